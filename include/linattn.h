@@ -1,0 +1,163 @@
+/*
+ * linattn.h -- C ABI of the B200 (sm_100a) ReLU linear-attention library.
+ *
+ * The operation is the linear attention of SANA-Video's Linear DiT, per
+ * attention head with head dimension d and phi = ReLU:
+ *
+ *   bidirectional (Eq. 2 with the rotary factors dropped, as the text under
+ *   Eq. 3 does):
+ *       S = sum_n phi(k_n)^T v_n   (d x d),   z = sum_n phi(k_n)   (d)
+ *       o_n = phi(q_n) S / (phi(q_n) . z + eps)
+ *
+ *   block-causal with the constant-memory cache (Eq. 3; Sec. 3.2 "KV Cache in
+ *   Block Linear Attention"; the cache update of Algorithm 1): tokens come in
+ *   contiguous blocks of frames; a block attends to itself and to every
+ *   earlier block.  The whole past is the running pair (sum S, sum phi(K)^T)
+ *   per head, kept in fp32; no per-token K/V is stored and the cache size
+ *   does not depend on the number of blocks (Table 1).
+ *
+ * Conventions common to every call
+ * --------------------------------
+ *  - All tensor pointers are DEVICE pointers.  The library never allocates or
+ *    frees device memory and never keeps a caller's pointer beyond what is
+ *    documented for the cache handle.  Descriptors, handles and out-params
+ *    are HOST memory.
+ *  - Q, K, V, O share one layout: element (b, n, h, e) is at element offset
+ *    b*stride_b + n*stride_n + h*stride_h + e.  A stride of 0 in the
+ *    descriptor selects the dense [B, N, H, d] default for that call's N.
+ *    Tokens are ordered frame-major, so a block of frames is a contiguous
+ *    token range.
+ *  - dtype LINATTN_BF16: Q, K, V, O are bfloat16; products are exact in fp32,
+ *    accumulation is fp32, O is rounded to nearest-even once at the store.
+ *    dtype LINATTN_F32: fp32 in and out, fp32 arithmetic.
+ *  - A "state" is, per (b, h), a (d+1) x d fp32 matrix W stored row-major,
+ *    units ordered [B][H]:   W[j][i] = S[i][j]  for j < d  (i: key feature,
+ *    j: value feature),      W[d][i] = z[i].
+ *    Its size is B*H*(d*d+d)*4 bytes.  It is plain memory: a copy of it is a
+ *    complete checkpoint of a stream.
+ *  - `stream` is a cudaStream_t passed as void* (NULL: the default stream).
+ *    Calls enqueue work and return; they do not synchronise.
+ *  - Pointers must be 16-byte aligned and strides multiples of 8 elements
+ *    (bf16) or 4 elements (fp32).  O must not alias Q, K or V.
+ *  - Every function returns LINATTN_OK (0) or a negative linattn_status.
+ *    Arguments are validated before anything is launched.  Zero tokens is a
+ *    successful no-op (linattn_state then writes a zero state; linattn_forward
+ *    writes nothing).  Nothing here throws, aborts or traps the device; the
+ *    only device-side wait (the grid barrier of the fused kernels) gives up
+ *    after a bounded number of polls and records LINATTN_ERR_TIMEOUT in the
+ *    workspace, readable with linattn_workspace_status.
+ *  - Calls that share a workspace (or a cache) must be ordered on one stream:
+ *    two of them in flight at once race on the split-N partials.
+ */
+#ifndef LINATTN_H_
+#define LINATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define LINATTN_API __attribute__((visibility("default")))
+#else
+#define LINATTN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum linattn_dtype { LINATTN_BF16 = 0, LINATTN_F32 = 1 } linattn_dtype;
+
+typedef enum linattn_status {
+  LINATTN_OK = 0,
+  LINATTN_ERR_INVALID_ARG = -1,        /* null pointer, negative size, bad enum, aliasing */
+  LINATTN_ERR_UNSUPPORTED = -2,        /* head dim outside 1..128, or a layout the kernels do not take */
+  LINATTN_ERR_BAD_ALIGNMENT = -3,      /* pointer or stride alignment rule above violated */
+  LINATTN_ERR_WORKSPACE_TOO_SMALL = -4,
+  LINATTN_ERR_CUDA = -5,               /* a CUDA runtime/driver call failed, or no sm_100 device */
+  LINATTN_ERR_TIMEOUT = -6,            /* a bounded device-side wait expired */
+  LINATTN_ERR_BAD_HANDLE = -7          /* cache handle is null, destroyed or corrupt */
+} linattn_status;
+
+/* Problem descriptor: plain data, filled by the caller, copied by the library. */
+typedef struct linattn_desc {
+  int32_t B;        /* batch */
+  int32_t H;        /* heads */
+  int32_t d;        /* head dimension, 1..128 (bf16 fast path: 32, 64, 112, 128) */
+  int32_t dtype;    /* linattn_dtype */
+  int64_t stride_b; /* element strides; 0 = dense [B,N,H,d] */
+  int64_t stride_n;
+  int64_t stride_h;
+} linattn_desc;
+
+LINATTN_API const char* linattn_status_string(int status);
+
+/* Bytes of one state for this descriptor: B*H*(d*d+d)*4 (Table 1's O(D^2) cache, per head). */
+LINATTN_API int linattn_state_bytes(const linattn_desc* desc, size_t* bytes);
+
+/* Scratch needed by linattn_forward / linattn_state for N tokens (split-N partial states and a
+ * small control block).  Depends on (B,H,d,dtype,N) only; works without a GPU. */
+LINATTN_API int linattn_workspace_bytes(const linattn_desc* desc, int64_t N, size_t* bytes);
+
+/* Zero a workspace's control block.  Call once after allocating a workspace (its first
+ * LINATTN_WORKSPACE_CTRL_BYTES bytes must start as zero) or to clear a recorded timeout. */
+#define LINATTN_WORKSPACE_CTRL_BYTES 4096
+LINATTN_API int linattn_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream`, then reports a device-side status recorded in the workspace
+ * (LINATTN_OK or LINATTN_ERR_TIMEOUT) through *status. */
+LINATTN_API int linattn_workspace_status(const void* workspace, void* stream, int* status);
+
+/* Eq. 2, whole sequence: O = phi(Q) S / (phi(Q) z + eps) with (S, z) reduced over all N tokens.
+ * q, k, v: in; o: out (same layout and dtype).  workspace: scratch, contents undefined after. */
+LINATTN_API int linattn_forward(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v, void* o,
+                    float eps, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The state of Eq. 2 / Eq. 3 alone: state = (sum_n phi(k_n)^T v_n, sum_n phi(k_n)) in the layout above.
+ * Deterministic: split-N partials are summed in a fixed order, so repeated calls give identical bits. */
+LINATTN_API int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void* v, float* state,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* The apply half of Eq. 2 alone: o_n = phi(q_n) S / (phi(q_n) . z + eps) for a given state. */
+LINATTN_API int linattn_apply(const linattn_desc* desc, int64_t N, const void* q, const float* state, void* o, float eps,
+                  void* stream);
+
+/* ---- block-causal form with the constant-memory cache (Eq. 3, Algorithm 1) ---- */
+
+typedef struct blocklin_cache blocklin_cache; /* opaque HOST handle */
+
+/* Sizes the caller must allocate on the device for a stream whose blocks have at most max_T_b
+ * tokens: the state (the cache proper; independent of max_T_b and of the number of blocks) and
+ * the scratch workspace. */
+LINATTN_API int blocklin_cache_bytes(const linattn_desc* desc, int64_t max_T_b, size_t* state_bytes, size_t* workspace_bytes);
+
+/* Create a handle over caller-owned device memory and enqueue zeroing of the state ("initialise
+ * the KV cache as empty", Algorithm 1).  The handle keeps the two device pointers; the caller
+ * keeps ownership and must keep them alive until blocklin_cache_destroy. */
+LINATTN_API int blocklin_cache_init(blocklin_cache** out, const linattn_desc* desc, float eps, void* dev_state,
+                        size_t state_bytes, void* dev_workspace, size_t workspace_bytes, void* stream);
+
+/* Forget the past: zero the state, blocks_seen = tokens_seen = 0. */
+LINATTN_API int blocklin_cache_reset(blocklin_cache* cache, void* stream);
+
+/* One block of T_b tokens ([B, T_b, H, d] with the descriptor's strides): add the block's own
+ * (S_blk, z_blk) to the cache, then apply the block's queries to the updated cache (the block
+ * attends to itself and to all earlier blocks).  o_blk and q_blk may both be NULL: absorb only. */
+LINATTN_API int blocklin_step(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
+                  void* o_blk, void* stream);
+
+/* n_blocks consecutive blocks of T_b tokens in one call over [B, n_blocks*T_b, H, d] tensors;
+ * result and final cache equal n_blocks calls of blocklin_step.  q and o may both be NULL. */
+LINATTN_API int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,
+                     const void* v, void* o, void* stream);
+
+/* Host-side bookkeeping; any out-param may be NULL. */
+LINATTN_API int blocklin_cache_info(const blocklin_cache* cache, int64_t* blocks_seen, int64_t* tokens_seen,
+                        size_t* state_bytes);
+
+/* Frees the host handle only; device memory stays the caller's. */
+LINATTN_API int blocklin_cache_destroy(blocklin_cache* cache);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LINATTN_H_ */

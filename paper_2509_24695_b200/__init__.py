@@ -1,0 +1,295 @@
+"""ReLU linear attention for B200 (sm_100a): thin Python binding of the C-ABI library.
+
+Every function here only marshals arguments (device pointers, sizes, strides, the
+current CUDA stream) into the ``extern "C"`` entry points declared in
+``include/linattn.h``; all arithmetic runs in the library's CUDA kernels.  PyTorch is
+used for device memory and streams only.  There is no CPU fallback: if the shared
+library cannot be loaded or built, or a call returns an error status, a
+``LinAttnError`` is raised.
+
+Tensors are ``[B, N, H, d]`` torch CUDA tensors (bfloat16 or float32) whose last axis
+is contiguous.  A state is a float32 tensor ``[B, H, d+1, d]``: rows ``0..d-1`` hold
+``S`` transposed (``state[b,h,j,i] = S[i,j]``), row ``d`` holds ``z``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+__all__ = [
+    "LinAttnError", "library_path", "load_library", "state_bytes", "workspace_bytes", "new_workspace",
+    "linattn_forward", "linattn_state", "linattn_apply", "split_state", "BlockLinCache", "workspace_status",
+]
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "liblinattn.so")
+
+LINATTN_BF16, LINATTN_F32 = 0, 1
+WORKSPACE_CTRL_BYTES = 4096
+
+
+class LinAttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib.linattn_status_string(status).decode() if _lib is not None else "library not loaded"
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+class _Desc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("d", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("stride_b", ctypes.c_int64), ("stride_n", ctypes.c_int64), ("stride_h", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library(path: str | None = None):
+    """Load ``liblinattn.so`` (building it in-tree with nvcc first if it is absent)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _LIB_PATH
+    if not os.path.exists(p):
+        from . import build as _build  # raises if nvcc fails: no fallback exists
+
+        p = _build.build()
+    lib = ctypes.CDLL(p)
+    vp, i64, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
+    dp = ctypes.POINTER(_Desc)
+    szp = ctypes.POINTER(sz)
+    f32 = ctypes.c_float
+    sig = {
+        "linattn_status_string": ([ctypes.c_int], ctypes.c_char_p),
+        "linattn_state_bytes": ([dp, szp], ctypes.c_int),
+        "linattn_workspace_bytes": ([dp, i64, szp], ctypes.c_int),
+        "linattn_workspace_init": ([vp, sz, vp], ctypes.c_int),
+        "linattn_workspace_status": ([vp, vp, ctypes.POINTER(ctypes.c_int)], ctypes.c_int),
+        "linattn_forward": ([dp, i64, vp, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
+        "linattn_state": ([dp, i64, vp, vp, vp, vp, sz, vp], ctypes.c_int),
+        "linattn_apply": ([dp, i64, vp, vp, vp, f32, vp], ctypes.c_int),
+        "blocklin_cache_bytes": ([dp, i64, szp, szp], ctypes.c_int),
+        "blocklin_cache_init": ([ctypes.POINTER(vp), dp, f32, vp, sz, vp, sz, vp], ctypes.c_int),
+        "blocklin_cache_reset": ([vp, vp], ctypes.c_int),
+        "blocklin_step": ([vp, i64, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_prefill": ([vp, i64, i64, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_cache_info": ([vp, ctypes.POINTER(i64), ctypes.POINTER(i64), szp], ctypes.c_int),
+        "blocklin_cache_destroy": ([vp], ctypes.c_int),
+    }
+    for name, (argtypes, restype) in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes, fn.restype = argtypes, restype
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise LinAttnError(status, where)
+
+
+def _torch():
+    import torch
+
+    return torch
+
+
+def _dtype_code(t) -> int:
+    torch = _torch()
+    if t.dtype == torch.bfloat16:
+        return LINATTN_BF16
+    if t.dtype == torch.float32:
+        return LINATTN_F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _desc_of(t, *same) -> _Desc:
+    """Descriptor for a [B, N, H, d] tensor; every tensor in `same` must share its layout."""
+    if t.dim() != 4 or t.stride(3) != 1 or not t.is_cuda:
+        raise ValueError("expected a CUDA tensor [B, N, H, d] with a contiguous last axis")
+    for o in same:
+        if o.shape != t.shape or o.stride() != t.stride() or o.dtype != t.dtype or o.device != t.device:
+            raise ValueError("q, k, v, o must share shape, strides, dtype and device")
+    B, N, H, d = t.shape
+    return _Desc(B, H, d, _dtype_code(t), t.stride(0), t.stride(1), t.stride(2))
+
+
+def _stream(t) -> int:
+    return _torch().cuda.current_stream(t.device).cuda_stream
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def state_bytes(B: int, H: int, d: int) -> int:
+    lib = load_library()
+    out = ctypes.c_size_t()
+    _check(lib.linattn_state_bytes(ctypes.byref(_Desc(B, H, d, 0, 0, 0, 0)), ctypes.byref(out)), "linattn_state_bytes")
+    return out.value
+
+
+def workspace_bytes(B: int, H: int, d: int, N: int, dtype_code: int = LINATTN_BF16) -> int:
+    lib = load_library()
+    out = ctypes.c_size_t()
+    _check(lib.linattn_workspace_bytes(ctypes.byref(_Desc(B, H, d, dtype_code, 0, 0, 0)), N, ctypes.byref(out)),
+           "linattn_workspace_bytes")
+    return out.value
+
+
+def new_workspace(like, N: int | None = None):
+    """Allocate (with torch) and initialise a workspace fit for tensors shaped like `like`."""
+    torch = _torch()
+    lib = load_library()
+    B, n, H, d = like.shape
+    nbytes = workspace_bytes(B, H, d, n if N is None else N, _dtype_code(like))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=like.device)
+    _check(lib.linattn_workspace_init(_ptr(ws), nbytes, _stream(like)), "linattn_workspace_init")
+    return ws
+
+
+def workspace_status(ws) -> int:
+    lib = load_library()
+    st = ctypes.c_int(0)
+    _check(lib.linattn_workspace_status(_ptr(ws), _stream(ws), ctypes.byref(st)), "linattn_workspace_status")
+    return st.value
+
+
+def linattn_forward(q, k, v, eps: float = 1e-6, out=None, workspace=None):
+    """Bidirectional ReLU linear attention (Eq. 2): returns O with the layout of q."""
+    torch = _torch()
+    lib = load_library()
+    o = torch.empty_like(q) if out is None else out
+    desc = _desc_of(q, k, v, o)
+    ws = new_workspace(q) if workspace is None else workspace
+    _check(lib.linattn_forward(ctypes.byref(desc), q.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o), eps,
+                               _ptr(ws), ws.numel(), _stream(q)), "linattn_forward")
+    return o
+
+
+def linattn_state(k, v, out=None, workspace=None):
+    """State of Eq. 2 / Eq. 3: float32 [B, H, d+1, d] (S transposed, then z)."""
+    torch = _torch()
+    lib = load_library()
+    desc = _desc_of(k, v)
+    B, N, H, d = k.shape
+    st = torch.empty((B, H, d + 1, d), dtype=torch.float32, device=k.device) if out is None else out
+    ws = new_workspace(k) if workspace is None else workspace
+    _check(lib.linattn_state(ctypes.byref(desc), N, _ptr(k), _ptr(v), _ptr(st), _ptr(ws), ws.numel(), _stream(k)),
+           "linattn_state")
+    return st
+
+
+def linattn_apply(q, state, eps: float = 1e-6, out=None):
+    """Apply half of Eq. 2 for a given state."""
+    torch = _torch()
+    lib = load_library()
+    o = torch.empty_like(q) if out is None else out
+    desc = _desc_of(q, o)
+    B, N, H, d = q.shape
+    if tuple(state.shape) != (B, H, d + 1, d) or state.dtype != torch.float32 or not state.is_contiguous():
+        raise ValueError("state must be a contiguous float32 [B, H, d+1, d] tensor")
+    _check(lib.linattn_apply(ctypes.byref(desc), N, _ptr(q), _ptr(state), _ptr(o), eps, _stream(q)), "linattn_apply")
+    return o
+
+
+def split_state(state):
+    """Views (S [B,H,d,d] indexed [key feature, value feature], z [B,H,d]) of a state tensor."""
+    d = state.shape[-1]
+    return state[..., :d, :].transpose(-1, -2), state[..., d, :]
+
+
+class BlockLinCache:
+    """Constant-memory cache of the block-causal form (Eq. 3, Algorithm 1's cache).
+
+    Owns (through torch) the fp32 state ``[B, H, d+1, d]`` and a scratch workspace; the
+    C handle only borrows their device pointers.  ``state`` is plain memory: cloning it
+    checkpoints the stream, copying into it restores one.
+    """
+
+    def __init__(self, B: int, H: int, d: int, dtype, device, max_T_b: int, eps: float = 1e-6,
+                 strides: tuple[int, int, int] = (0, 0, 0)):
+        torch = _torch()
+        self._lib = load_library()
+        code = LINATTN_BF16 if dtype == torch.bfloat16 else LINATTN_F32 if dtype == torch.float32 else None
+        if code is None:
+            raise TypeError(f"unsupported dtype {dtype}")
+        self._desc = _Desc(B, H, d, code, *strides)
+        sb, wb = ctypes.c_size_t(), ctypes.c_size_t()
+        _check(self._lib.blocklin_cache_bytes(ctypes.byref(self._desc), max_T_b, ctypes.byref(sb), ctypes.byref(wb)),
+               "blocklin_cache_bytes")
+        self.state = torch.empty((B, H, d + 1, d), dtype=torch.float32, device=device)
+        assert self.state.numel() * 4 == sb.value
+        self.workspace = torch.empty(wb.value, dtype=torch.uint8, device=device)
+        self.max_T_b = max_T_b
+        self._handle = ctypes.c_void_p()
+        _check(self._lib.blocklin_cache_init(ctypes.byref(self._handle), ctypes.byref(self._desc), eps,
+                                             _ptr(self.state), sb.value, _ptr(self.workspace), wb.value,
+                                             _stream(self.state)), "blocklin_cache_init")
+
+    def reset(self):
+        _check(self._lib.blocklin_cache_reset(self._handle, _stream(self.state)), "blocklin_cache_reset")
+
+    def step(self, q, k, v, out=None):
+        """cache += state(block); returns the block's output (None when q is None)."""
+        torch = _torch()
+        o = None
+        if q is not None:
+            o = torch.empty_like(q) if out is None else out
+            _desc_of(q, k, v, o)
+        else:
+            _desc_of(k, v)
+        self._check_layout(k)
+        _check(self._lib.blocklin_step(self._handle, k.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o), _stream(k)),
+               "blocklin_step")
+        return o
+
+    def prefill(self, q, k, v, n_blocks: int, out=None):
+        """n_blocks equal blocks in one call over [B, n_blocks*T_b, H, d] tensors."""
+        torch = _torch()
+        N = k.shape[1]
+        if n_blocks <= 0 or N % n_blocks:
+            raise ValueError("token count must be n_blocks * T_b")
+        o = None
+        if q is not None:
+            o = torch.empty_like(q) if out is None else out
+            _desc_of(q, k, v, o)
+        else:
+            _desc_of(k, v)
+        self._check_layout(k)
+        _check(self._lib.blocklin_prefill(self._handle, n_blocks, N // n_blocks, _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                                          _stream(k)), "blocklin_prefill")
+        return o
+
+    def _check_layout(self, t):
+        """The cache's descriptor fixes (B, H, d, dtype, strides); a block must match it."""
+        dsc = self._desc
+        if (t.shape[0], t.shape[2], t.shape[3]) != (dsc.B, dsc.H, dsc.d) or _dtype_code(t) != dsc.dtype:
+            raise ValueError("block does not match the cache's (B, H, d, dtype)")
+        want = (dsc.stride_b, dsc.stride_n, dsc.stride_h)
+        if want == (0, 0, 0):
+            if not t.is_contiguous():
+                raise ValueError("this cache was created for dense [B, T_b, H, d] blocks")
+        elif t.numel() and tuple(t.stride()[:3]) != want:
+            raise ValueError(f"block strides {tuple(t.stride()[:3])} differ from the cache's {want}")
+
+    def info(self) -> dict:
+        b, t, s = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_size_t()
+        _check(self._lib.blocklin_cache_info(self._handle, ctypes.byref(b), ctypes.byref(t), ctypes.byref(s)),
+               "blocklin_cache_info")
+        return {"blocks_seen": b.value, "tokens_seen": t.value, "state_bytes": s.value}
+
+    def close(self):
+        if self._handle:
+            self._lib.blocklin_cache_destroy(self._handle)
+            self._handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,301 @@
+// C ABI of the linear-attention library: argument validation, workspace layout, kernel selection
+// and the host-side cache handle.  See include/linattn.h for the contract of each entry point.
+#include <new>
+
+#include "common.cuh"
+
+using namespace linattn;
+
+namespace {
+
+constexpr uint32_t kCacheMagic = 0x4C41434Bu;  // "LACK"
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates a descriptor and resolves its strides for N tokens.
+int resolve(const linattn_desc* desc, long long N, Problem* out) {
+  if (!desc || N < 0) return LINATTN_ERR_INVALID_ARG;
+  if (desc->B < 1 || desc->H < 1 || desc->d < 1) return LINATTN_ERR_INVALID_ARG;
+  if (desc->dtype != LINATTN_BF16 && desc->dtype != LINATTN_F32) return LINATTN_ERR_INVALID_ARG;
+  if (desc->stride_b < 0 || desc->stride_n < 0 || desc->stride_h < 0) return LINATTN_ERR_INVALID_ARG;
+  if (desc->d > 128) return LINATTN_ERR_UNSUPPORTED;
+  if ((long long)desc->B * desc->H > 65535) return LINATTN_ERR_UNSUPPORTED;
+  Problem p;
+  p.B = desc->B; p.H = desc->H; p.d = desc->d; p.dtype = desc->dtype; p.N = N;
+  p.sh = desc->stride_h ? desc->stride_h : desc->d;
+  p.sn = desc->stride_n ? desc->stride_n : (long long)desc->H * desc->d;
+  p.sb = desc->stride_b ? desc->stride_b : (long long)N * desc->H * desc->d;
+  if (p.sh < p.d) return LINATTN_ERR_INVALID_ARG;
+  *out = p;
+  return LINATTN_OK;
+}
+
+// Alignment rule of the header: 16-byte pointers, strides multiples of 16 bytes.  Enforced for the
+// shapes the tensor-core kernels take (their TMA descriptors need it); the FMA kernels use scalar
+// accesses and only need natural alignment.
+int check_alignment(const Problem& p, const void* a, const void* b, const void* c, const void* d) {
+  if (!umma_supported(p)) return LINATTN_OK;
+  const void* ptrs[4] = {a, b, c, d};
+  for (const void* x : ptrs)
+    if (x && !aligned16(x)) return LINATTN_ERR_BAD_ALIGNMENT;
+  if ((p.sb % 8) || (p.sn % 8) || (p.sh % 8)) return LINATTN_ERR_BAD_ALIGNMENT;
+  return LINATTN_OK;
+}
+
+size_t partial_bytes(const Problem& p) {
+  if (umma_supported(p)) return umma_partial_bytes(p);
+  return sizeof(float) * (size_t)p.state_elems() * p.units() * fma_chunks(p.N);
+}
+
+inline size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+inline size_t state_bytes_of(const Problem& p) { return sizeof(float) * (size_t)p.state_elems() * p.units(); }
+
+// Workspace layout: [control block][split-N partials][one state, used by linattn_forward].
+size_t state_slot_offset(const Problem& p) { return round256(LINATTN_WORKSPACE_CTRL_BYTES + partial_bytes(p)); }
+
+size_t workspace_need(const Problem& p) { return round256(state_slot_offset(p) + state_bytes_of(p)); }
+
+inline float* partials_of(void* workspace) {
+  return reinterpret_cast<float*>(static_cast<char*>(workspace) + LINATTN_WORKSPACE_CTRL_BYTES);
+}
+
+int cuda_status(cudaError_t e) { return e == cudaSuccess ? LINATTN_OK : LINATTN_ERR_CUDA; }
+
+// state_out = (accumulate ? state_out : 0) + state(k, v)
+int run_state(const Problem& p, const void* k, const void* v, float* state, bool accumulate, void* workspace,
+              cudaStream_t stream) {
+  if (umma_supported(p)) return umma_state(p, k, v, state, accumulate, workspace, stream);
+  return cuda_status(fma_state(p, k, v, state, accumulate, partials_of(workspace), stream));
+}
+
+int run_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream) {
+  if (umma_supported(p)) return umma_apply(p, q, state, o, eps, stream);
+  return cuda_status(fma_apply(p, q, state, o, eps, stream));
+}
+
+}  // namespace
+
+struct blocklin_cache {
+  uint32_t magic;
+  linattn_desc desc;
+  float eps;
+  float* state;
+  size_t state_bytes;
+  void* workspace;
+  size_t workspace_bytes;
+  long long blocks_seen;
+  long long tokens_seen;
+};
+
+// One block: commit (cache += (S_blk, z_blk)), then read (the block's queries see the updated cache).
+static int step_impl(blocklin_cache* cache, const Problem& p, const void* q_blk, const void* k_blk,
+                     const void* v_blk, void* o_blk, cudaStream_t stream) {
+  if ((q_blk == nullptr) != (o_blk == nullptr)) return LINATTN_ERR_INVALID_ARG;
+  if (p.N > 0 && (!k_blk || !v_blk)) return LINATTN_ERR_INVALID_ARG;
+  if (o_blk && (o_blk == q_blk || o_blk == k_blk || o_blk == v_blk)) return LINATTN_ERR_INVALID_ARG;
+  int st = check_alignment(p, q_blk, k_blk, v_blk, o_blk);
+  if (st != LINATTN_OK) return st;
+  if (cache->workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  if (p.N == 0) return LINATTN_OK;
+  st = run_state(p, k_blk, v_blk, cache->state, true, cache->workspace, stream);
+  if (st != LINATTN_OK) return st;
+  if (q_blk) {
+    st = run_apply(p, q_blk, cache->state, o_blk, cache->eps, stream);
+    if (st != LINATTN_OK) return st;
+  }
+  cache->blocks_seen += 1;
+  cache->tokens_seen += p.N;
+  return LINATTN_OK;
+}
+
+extern "C" {
+
+const char* linattn_status_string(int status) {
+  switch (status) {
+    case LINATTN_OK: return "ok";
+    case LINATTN_ERR_INVALID_ARG: return "invalid argument";
+    case LINATTN_ERR_UNSUPPORTED: return "unsupported shape or layout";
+    case LINATTN_ERR_BAD_ALIGNMENT: return "pointer or stride not 16-byte aligned";
+    case LINATTN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case LINATTN_ERR_CUDA: return "CUDA call failed";
+    case LINATTN_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case LINATTN_ERR_BAD_HANDLE: return "bad cache handle";
+    default: return "unknown status";
+  }
+}
+
+int linattn_state_bytes(const linattn_desc* desc, size_t* bytes) {
+  Problem p;
+  if (!bytes) return LINATTN_ERR_INVALID_ARG;
+  int st = resolve(desc, 0, &p);
+  if (st != LINATTN_OK) return st;
+  *bytes = sizeof(float) * (size_t)p.state_elems() * p.units();
+  return LINATTN_OK;
+}
+
+int linattn_workspace_bytes(const linattn_desc* desc, int64_t N, size_t* bytes) {
+  Problem p;
+  if (!bytes) return LINATTN_ERR_INVALID_ARG;
+  int st = resolve(desc, N, &p);
+  if (st != LINATTN_OK) return st;
+  *bytes = workspace_need(p);
+  return LINATTN_OK;
+}
+
+int linattn_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace || workspace_bytes < LINATTN_WORKSPACE_CTRL_BYTES) return LINATTN_ERR_INVALID_ARG;
+  return cuda_status(cudaMemsetAsync(workspace, 0, LINATTN_WORKSPACE_CTRL_BYTES, (cudaStream_t)stream));
+}
+
+int linattn_workspace_status(const void* workspace, void* stream, int* status) {
+  if (!workspace || !status) return LINATTN_ERR_INVALID_ARG;
+  int word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return LINATTN_ERR_CUDA;
+  *status = word;
+  return LINATTN_OK;
+}
+
+int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void* v, float* state, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+  Problem p;
+  int st = resolve(desc, N, &p);
+  if (st != LINATTN_OK) return st;
+  if (!state || !workspace) return LINATTN_ERR_INVALID_ARG;
+  if (N > 0 && (!k || !v)) return LINATTN_ERR_INVALID_ARG;
+  if ((st = check_alignment(p, k, v, state, workspace)) != LINATTN_OK) return st;
+  if (workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  return run_state(p, k, v, state, false, workspace, (cudaStream_t)stream);
+}
+
+int linattn_apply(const linattn_desc* desc, int64_t N, const void* q, const float* state, void* o, float eps,
+                  void* stream) {
+  Problem p;
+  int st = resolve(desc, N, &p);
+  if (st != LINATTN_OK) return st;
+  if (!state) return LINATTN_ERR_INVALID_ARG;
+  if (N > 0 && (!q || !o || q == o)) return LINATTN_ERR_INVALID_ARG;
+  if ((st = check_alignment(p, q, o, state, nullptr)) != LINATTN_OK) return st;
+  return run_apply(p, q, state, o, eps, (cudaStream_t)stream);
+}
+
+int linattn_forward(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v, void* o,
+                    float eps, void* workspace, size_t workspace_bytes, void* stream) {
+  Problem p;
+  int st = resolve(desc, N, &p);
+  if (st != LINATTN_OK) return st;
+  if (!workspace) return LINATTN_ERR_INVALID_ARG;
+  if (N > 0 && (!q || !k || !v || !o || o == q || o == k || o == v)) return LINATTN_ERR_INVALID_ARG;
+  if ((st = check_alignment(p, q, k, v, o)) != LINATTN_OK) return st;
+  if (!aligned16(workspace)) return LINATTN_ERR_BAD_ALIGNMENT;
+  if (workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  if (N == 0) return LINATTN_OK;
+  // the forward keeps its reduced state in the workspace, after the partials
+  float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + state_slot_offset(p));
+  st = run_state(p, k, v, state, false, workspace, (cudaStream_t)stream);
+  if (st != LINATTN_OK) return st;
+  return run_apply(p, q, state, o, eps, (cudaStream_t)stream);
+}
+
+int blocklin_cache_bytes(const linattn_desc* desc, int64_t max_T_b, size_t* state_bytes, size_t* workspace_bytes) {
+  Problem p;
+  int st = resolve(desc, max_T_b, &p);
+  if (st != LINATTN_OK) return st;
+  if (!state_bytes || !workspace_bytes) return LINATTN_ERR_INVALID_ARG;
+  *state_bytes = sizeof(float) * (size_t)p.state_elems() * p.units();
+  *workspace_bytes = workspace_need(p);
+  return LINATTN_OK;
+}
+
+int blocklin_cache_init(blocklin_cache** out, const linattn_desc* desc, float eps, void* dev_state,
+                        size_t state_bytes, void* dev_workspace, size_t workspace_bytes, void* stream) {
+  if (!out) return LINATTN_ERR_INVALID_ARG;
+  *out = nullptr;
+  Problem p;
+  int st = resolve(desc, 0, &p);
+  if (st != LINATTN_OK) return st;
+  if (!dev_state || !dev_workspace) return LINATTN_ERR_INVALID_ARG;
+  if (!aligned16(dev_state) || !aligned16(dev_workspace)) return LINATTN_ERR_BAD_ALIGNMENT;
+  const size_t need_state = state_bytes_of(p);
+  if (state_bytes < need_state) return LINATTN_ERR_INVALID_ARG;
+  if (workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  blocklin_cache* c = new (std::nothrow) blocklin_cache;
+  if (!c) return LINATTN_ERR_INVALID_ARG;
+  c->magic = kCacheMagic;
+  c->desc = *desc;
+  c->eps = eps;
+  c->state = static_cast<float*>(dev_state);
+  c->state_bytes = need_state;
+  c->workspace = dev_workspace;
+  c->workspace_bytes = workspace_bytes;
+  c->blocks_seen = 0;
+  c->tokens_seen = 0;
+  cudaError_t e = cudaMemsetAsync(dev_state, 0, need_state, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(dev_workspace, 0, LINATTN_WORKSPACE_CTRL_BYTES, (cudaStream_t)stream);
+  if (e != cudaSuccess) {
+    c->magic = 0;
+    delete c;
+    return LINATTN_ERR_CUDA;
+  }
+  *out = c;
+  return LINATTN_OK;
+}
+
+int blocklin_cache_reset(blocklin_cache* cache, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  cache->blocks_seen = 0;
+  cache->tokens_seen = 0;
+  return cuda_status(cudaMemsetAsync(cache->state, 0, cache->state_bytes, (cudaStream_t)stream));
+}
+
+int blocklin_step(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
+                  void* o_blk, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  Problem p;
+  int st = resolve(&cache->desc, T_b, &p);
+  if (st != LINATTN_OK) return st;
+  return step_impl(cache, p, q_blk, k_blk, v_blk, o_blk, (cudaStream_t)stream);
+}
+
+int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,
+                     const void* v, void* o, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  if (n_blocks < 0 || T_b < 0) return LINATTN_ERR_INVALID_ARG;
+  if ((q == nullptr) != (o == nullptr)) return LINATTN_ERR_INVALID_ARG;
+  if (n_blocks == 0 || T_b == 0) return LINATTN_OK;
+  if (!k || !v) return LINATTN_ERR_INVALID_ARG;
+  // The tensors are [B, n_blocks*T_b, H, d]; block i is the token range [i*T_b, (i+1)*T_b) of each batch
+  // entry, so every block keeps the whole sequence's strides.
+  Problem p;
+  int st = resolve(&cache->desc, n_blocks * T_b, &p);
+  if (st != LINATTN_OK) return st;
+  p.N = T_b;
+  const size_t esz = cache->desc.dtype == LINATTN_BF16 ? 2 : 4;
+  for (int64_t i = 0; i < n_blocks && st == LINATTN_OK; ++i) {
+    const size_t off = (size_t)(i * T_b) * (size_t)p.sn * esz;
+    st = step_impl(cache, p, q ? static_cast<const char*>(q) + off : nullptr, static_cast<const char*>(k) + off,
+                   static_cast<const char*>(v) + off, o ? static_cast<char*>(o) + off : nullptr,
+                   (cudaStream_t)stream);
+  }
+  return st;
+}
+
+int blocklin_cache_info(const blocklin_cache* cache, int64_t* blocks_seen, int64_t* tokens_seen,
+                        size_t* state_bytes) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  if (blocks_seen) *blocks_seen = cache->blocks_seen;
+  if (tokens_seen) *tokens_seen = cache->tokens_seen;
+  if (state_bytes) *state_bytes = cache->state_bytes;
+  return LINATTN_OK;
+}
+
+int blocklin_cache_destroy(blocklin_cache* cache) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  cache->magic = 0;
+  delete cache;
+  return LINATTN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,55 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "linattn.h"
+
+namespace linattn {
+
+// A descriptor with its strides resolved for one call.
+struct Problem {
+  int B, H, d;
+  int dtype;
+  long long sb, sn, sh;  // element strides of (batch, token, head); the feature axis is contiguous
+  long long N;           // tokens in this call
+  __host__ __device__ int units() const { return B * H; }
+  __host__ __device__ long long state_elems() const { return (long long)(d + 1) * d; }  // floats per (b,h) state
+};
+
+// Control block at the start of every workspace.
+struct WorkspaceCtrl {
+  int status;            // LINATTN_OK or LINATTN_ERR_TIMEOUT, written by kernels
+  int pad0[15];
+  unsigned barrier[16];  // grid-barrier counters of the fused kernels
+  unsigned unit_arrivals[960];
+};
+static_assert(sizeof(WorkspaceCtrl) <= LINATTN_WORKSPACE_CTRL_BYTES, "control block too large");
+
+constexpr int kMaxCtas = 256;        // upper bound on the persistent grid (B200 has 148 SMs)
+constexpr int kFmaMaxChunks = 64;    // split-N partials per unit on the FMA path
+constexpr int kFmaMinChunkTokens = 512;
+
+inline int fma_chunks(long long N) {
+  long long p = (N + kFmaMinChunkTokens - 1) / kFmaMinChunkTokens;
+  if (p < 1) p = 1;
+  return p > kFmaMaxChunks ? kFmaMaxChunks : (int)p;
+}
+
+// ---- FMA kernels (fp32 I/O path, and bf16 shapes the tensor-core kernels do not take) ----
+// state_out = (accumulate ? state_out : 0) + state of tokens [0, N); partials is scratch.
+cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate,
+                      float* partials, cudaStream_t stream);
+cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream);
+
+// ---- tensor-core (tcgen05 + TMA) kernels, bf16, d in {32, 64, 112, 128} ----
+bool umma_supported(const Problem& p);
+size_t umma_partial_bytes(const Problem& p);
+// Returns LINATTN_OK or an error status.
+int umma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate, void* workspace,
+               cudaStream_t stream);
+int umma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream);
+
+}  // namespace linattn

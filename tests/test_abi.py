@@ -1,0 +1,81 @@
+"""The C-ABI shared library: it builds for sm_100a, loads without a GPU, exports every symbol the
+public header declares, and its host-side validation answers without touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2509_24695_b200 import build, load_library
+
+    build.build()
+    return load_library()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "linattn.h")).read()
+    return sorted(set(re.findall(r"LINATTN_API\s+[\w\s\*]+?\b((?:linattn|blocklin)_\w+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    names = declared_symbols()
+    assert {"linattn_forward", "linattn_state", "linattn_apply", "blocklin_cache_init", "blocklin_cache_reset",
+            "blocklin_step", "blocklin_prefill"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in linattn.h but not exported"
+
+
+def test_header_compiles_as_plain_c(tmp_path):
+    import subprocess
+
+    src = tmp_path / "t.c"
+    src.write_text('#include "linattn.h"\nint main(void){ linattn_desc d; (void)d; return LINATTN_OK; }\n')
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), "-c", str(src),
+                           "-o", str(tmp_path / "t.o")])
+
+
+def test_sizes_and_validation_without_gpu(lib):
+    import paper_2509_24695_b200 as la
+
+    # Table 1: the cache is O(d^2) per head and nothing else
+    assert la.state_bytes(1, 20, 112) == 20 * (112 * 112 + 112) * 4 == 1012480
+    assert la.state_bytes(2, 20, 112) == 2024960
+    w1 = la.workspace_bytes(1, 20, 112, 32760)
+    assert w1 >= la.WORKSPACE_CTRL_BYTES + 1012480 and w1 % 256 == 0
+    assert la.workspace_bytes(1, 20, 112, 0) >= la.WORKSPACE_CTRL_BYTES
+    for args, status in [((0, 20, 112, 10), -1), ((1, 20, 0, 10), -1), ((1, 20, 129, 10), -2), ((1, 20, 112, -1), -1)]:
+        with pytest.raises(la.LinAttnError) as e:
+            la.workspace_bytes(*args)
+        assert e.value.status == status
+    assert lib.linattn_status_string(0) == b"ok"
+    assert b"workspace" in lib.linattn_status_string(-4)
+    # null pointers are rejected before any launch
+    d = la._Desc(1, 2, 112, 0, 0, 0, 0)
+    assert lib.linattn_forward(ctypes.byref(d), 8, None, None, None, None, 1e-6, None, 0, None) == -1
+    assert lib.linattn_forward(None, 8, None, None, None, None, 1e-6, None, 0, None) == -1
+    assert lib.blocklin_step(None, 8, None, None, None, None, None) == -7
+    assert lib.blocklin_cache_reset(None, None) == -7
+    assert lib.blocklin_cache_destroy(None) == -7
+    sb, wb = ctypes.c_size_t(), ctypes.c_size_t()
+    assert lib.blocklin_cache_bytes(ctypes.byref(d), 4680, ctypes.byref(sb), ctypes.byref(wb)) == 0
+    assert sb.value == 2 * (112 * 112 + 112) * 4
+    h = ctypes.c_void_p()
+    assert lib.blocklin_cache_init(ctypes.byref(h), ctypes.byref(d), 1e-6, None, sb.value, None, wb.value, None) == -1
+    assert not h.value
+
+
+def test_product_package_does_not_touch_the_oracle():
+    """The oracle is test infrastructure: nothing under the package may import or load it."""
+    pkg = os.path.join(ROOT, "paper_2509_24695_b200")
+    for dirpath, _, files in os.walk(pkg):
+        if "_build" in dirpath:
+            continue
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".c", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "from oracle" not in text and "liblinattn_oracle" not in text, f

@@ -1,0 +1,192 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle, element by element,
+on the same seeded inputs.  Sizes here span several tiles and ragged tails but stay small enough
+for the oracle to finish in seconds; the full-size workloads are in test_gpu_fullsize.py."""
+import numpy as np
+import pytest
+
+from paper_2509_24695_b200 import synth
+from parity_util import assert_parity_bf16, assert_parity_f32, assert_state_close, to_dev, to_f64
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-6
+
+
+@pytest.fixture(scope="module")
+def la():
+    import torch
+
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    import paper_2509_24695_b200 as la
+
+    la.load_library()
+    return la
+
+
+def gen(B, N, H, d, seed, dtype, scale=1.0):
+    return tuple(synth.gauss((B, N, H, d), seed, t, scale=scale, dtype=dtype) for t in (1, 2, 3))
+
+
+def check(dtype, got, ref, what):
+    (assert_parity_bf16 if dtype == "bf16" else assert_parity_f32)(got, ref, what)
+
+
+SHAPES = [
+    # B, N, H, d
+    (1, 192, 4, 32),      # config 1
+    (2, 1000, 3, 112),    # several 128-token tiles + ragged tail, the paper's head dim
+    (1, 129, 2, 112),
+    (1, 127, 2, 112),
+    (1, 1, 1, 112),
+    (1, 2, 5, 64),
+    (2, 777, 5, 64),
+    (1, 515, 7, 32),      # head count not a multiple of the 4-head packing
+    (2, 300, 3, 128),
+    (1, 333, 2, 16),      # head dims outside the tensor-core set
+    (1, 77, 3, 7),
+    (1, 260, 1, 96),
+]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "B%d_N%d_H%d_d%d" % s)
+def test_forward_matches_oracle(la, orc, shape, dtype):
+    B, N, H, d = shape
+    q, k, v = gen(B, N, H, d, 2000 + N + d, dtype)
+    ref = orc.forward(q, k, v, EPS)
+    o = la.linattn_forward(to_dev(q), to_dev(k), to_dev(v), EPS)
+    check(dtype, to_f64(o), ref, f"forward {shape} {dtype}")
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("shape", [(2, 1000, 3, 112), (1, 515, 7, 32), (2, 300, 3, 128), (1, 77, 3, 7)],
+                         ids=lambda s: "B%d_N%d_H%d_d%d" % s)
+def test_state_and_apply_match_oracle(la, orc, shape, dtype):
+    import torch
+
+    B, N, H, d = shape
+    q, k, v = gen(B, N, H, d, 2100 + N + d, dtype)
+    S, z = orc.state(k, v)
+    st = la.linattn_state(to_dev(k), to_dev(v))
+    assert tuple(st.shape) == (B, H, d + 1, d) and st.dtype == torch.float32
+    assert_state_close(to_f64(st), S, z, 1e-5, f"state {shape} {dtype}")
+    # apply the ORACLE's state (rounded to fp32) so this checks the apply half alone
+    W = np.concatenate([S.swapaxes(-1, -2), z[..., None, :]], axis=-2).astype(np.float32)
+    o = la.linattn_apply(to_dev(q), torch.from_numpy(W).cuda(), EPS)
+    ref = orc.apply_rows(q, W[..., :d, :].swapaxes(-1, -2).astype(np.float64).copy(), W[..., d, :].astype(np.float64).copy(),
+                         EPS, np.arange(N))
+    check(dtype, to_f64(o), ref, f"apply {shape} {dtype}")
+
+
+@pytest.mark.parametrize("shape", [(2, 1000, 3, 112), (1, 515, 7, 32), (1, 4097, 2, 64), (1, 300, 2, 128)],
+                         ids=lambda s: "B%d_N%d_H%d_d%d" % s)
+def test_integer_inputs_give_bit_exact_state(la, orc, shape):
+    """Inputs in {-2..2}: every partial sum is an integer < 2^24, so fp32 accumulation in any order
+    must reproduce the oracle's state bit for bit (no tile lost, none counted twice)."""
+    B, N, H, d = shape
+    k = synth.smallint(shape[:1] + (N, H, d), 31, 2, 2)
+    v = synth.smallint(shape[:1] + (N, H, d), 31, 3, 2)
+    S, z = orc.state(k, v)
+    st = to_f64(la.linattn_state(to_dev(k), to_dev(v)))
+    assert np.array_equal(st[..., :d, :].swapaxes(-1, -2), S)
+    assert np.array_equal(st[..., d, :], z)
+
+
+def test_run_to_run_determinism(la):
+    import torch
+
+    q, k, v = (to_dev(x) for x in gen(2, 3000, 3, 112, 77, "bf16"))
+    ws = la.new_workspace(q)
+    o1 = la.linattn_forward(q, k, v, EPS, workspace=ws).clone()
+    s1 = la.linattn_state(k, v, workspace=ws).clone()
+    for _ in range(3):
+        assert torch.equal(la.linattn_forward(q, k, v, EPS, workspace=ws), o1)
+        assert torch.equal(la.linattn_state(k, v, workspace=ws), s1)
+
+
+@pytest.mark.parametrize("d", [112, 32])
+def test_constant_v_outputs_are_order_one(la, orc, d):
+    """v_n = c: o = c*D/(D+eps).  Outputs of size ~1, so the absolute tolerance term is not vacuous."""
+    B, N, H = 1, 700, 3
+    q, k, _ = gen(B, N, H, d, 88, "bf16")
+    c = synth.gauss((d,), 89, 3, dtype="bf16")
+    v = np.broadcast_to(c, (B, N, H, d)).copy()
+    o = to_f64(la.linattn_forward(to_dev(q), to_dev(k), to_dev(v), EPS))
+    ref = orc.forward(q, k, v, EPS)
+    assert_parity_bf16(o, ref, "constant V")
+    cf = synth.bf16_bits_to_f32(c).astype(np.float64)
+    live = np.abs(ref).sum(axis=-1) > 0
+    assert np.allclose(o[live], np.broadcast_to(cf, o.shape)[live], rtol=1e-2, atol=1e-2)
+
+
+@pytest.mark.parametrize("d", [112, 64])
+def test_one_hot_features_give_segment_means(la, orc, d):
+    B, N, H, C = 1, 900, 2, 5
+    a = synth.index((N,), 91, 1, C)
+    c = synth.index((N,), 91, 2, C)
+    q = np.zeros((B, N, H, d), np.float32); q[0, np.arange(N), :, a * 3] = 1.0
+    k = np.zeros((B, N, H, d), np.float32); k[0, np.arange(N), :, c * 3] = 2.0
+    v = synth.bf16_bits_to_f32(synth.smallint((B, N, H, d), 91, 3, 4))
+    qb, kb, vb = (synth.f32_to_bf16_bits(x) for x in (q, k, v))
+    o = to_f64(la.linattn_forward(to_dev(qb), to_dev(kb), to_dev(vb), EPS))
+    ref = orc.forward(qb, kb, vb, EPS)
+    assert_parity_bf16(o, ref, "one-hot")
+    cnt = np.bincount(c, minlength=C)
+    mean = np.stack([np.bincount(c, weights=v[0, :, 0, j].astype(np.float64), minlength=C) / cnt for j in range(4)], 1)
+    assert np.allclose(o[0, :, 0, :4], mean[a], rtol=1e-2, atol=1e-2)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_dead_queries_give_exact_zero(la, orc, dtype):
+    """A query row with no positive entry has phi(q).z = 0: the output is 0/(0+eps) = 0, never NaN."""
+    import torch
+
+    B, N, H, d = 1, 300, 2, 112
+    q, k, v = gen(B, N, H, d, 93, "f32")
+    q[0, 5] = -np.abs(q[0, 5]); q[0, 128] = 0.0; q[0, 299, 1] = -1.0
+    if dtype == "bf16":
+        q, k, v = (synth.f32_to_bf16_bits(x) for x in (q, k, v))
+    o = la.linattn_forward(to_dev(q), to_dev(k), to_dev(v), EPS)
+    assert torch.isfinite(o.float()).all()
+    assert (o[0, 5] == 0).all() and (o[0, 128] == 0).all() and (o[0, 299, 1] == 0).all()
+    check(dtype, to_f64(o), orc.forward(q, k, v, EPS), "dead queries")
+    # empty state: all keys non-positive -> every output is exactly zero
+    k2 = -np.abs(synth.gauss((B, N, H, d), 94, 2, dtype="f32"))
+    k2 = synth.f32_to_bf16_bits(k2) if dtype == "bf16" else k2
+    o2 = la.linattn_forward(to_dev(q), to_dev(k2), to_dev(v), EPS)
+    assert (o2 == 0).all()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_head_major_strides(la, orc, dtype):
+    """[B,H,N,d] storage passed as a [B,N,H,d] view."""
+    B, N, H, d = 2, 400, 3, 112
+    q, k, v = gen(B, N, H, d, 95, dtype)
+    ref = orc.forward(q, k, v, EPS)
+    hm = lambda x: to_dev(np.ascontiguousarray(x.transpose(0, 2, 1, 3))).permute(0, 2, 1, 3)
+    o = la.linattn_forward(hm(q), hm(k), hm(v), EPS)
+    assert o.stride() == hm(q).stride()
+    check(dtype, to_f64(o), ref, "head-major")
+
+
+def test_zero_tokens_and_errors(la):
+    import torch
+
+    q = torch.zeros((1, 0, 2, 112), dtype=torch.bfloat16, device="cuda")
+    o = la.linattn_forward(q, q.clone(), q.clone(), EPS)
+    assert o.shape == q.shape
+    st = la.linattn_state(q, q.clone())
+    assert (st == 0).all()
+    x = torch.zeros((1, 8, 2, 112), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(la.LinAttnError) as e:
+        la.linattn_forward(x, x, x, EPS, out=x)  # aliasing
+    assert e.value.status == -1
+    big = torch.zeros((1, 8, 1, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(la.LinAttnError) as e:
+        la.linattn_forward(big, big.clone(), big.clone(), EPS)
+    assert e.value.status == -2
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    with pytest.raises(la.LinAttnError) as e:
+        la.linattn_forward(x, x.clone(), x.clone(), EPS, workspace=ws)
+    assert e.value.status == -4
+    assert la.workspace_status(la.new_workspace(x)) == 0
