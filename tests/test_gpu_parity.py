@@ -71,7 +71,7 @@ def test_state_and_apply_match_oracle(la, orc, shape, dtype):
     assert tuple(st.shape) == (B, H, d + 1, d) and st.dtype == torch.float32
     assert_state_close(to_f64(st), S, z, 1e-5, f"state {shape} {dtype}")
     # apply the ORACLE's state (rounded to fp32) so this checks the apply half alone
-    W = np.concatenate([S.swapaxes(-1, -2), z[..., None, :]], axis=-2).astype(np.float32)
+    W = np.ascontiguousarray(np.concatenate([S.swapaxes(-1, -2), z[..., None, :]], axis=-2), dtype=np.float32)
     o = la.linattn_apply(to_dev(q), torch.from_numpy(W).cuda(), EPS)
     ref = orc.apply_rows(q, W[..., :d, :].swapaxes(-1, -2).astype(np.float64).copy(), W[..., d, :].astype(np.float64).copy(),
                          EPS, np.arange(N))
