@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the ReLU linear-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 480p|720p]
+
+One step = one pass of the bidirectional hot path (state reduction over K,V + apply over Q, writing
+bf16 O) over one batch of seeded synthetic input shaped like a 480p 5-second latent (20 heads x 112,
+32760 tokens).  The metric is linear-attention tokens*heads per second.  Rank 0 prints ONE JSON line.
+
+`--impl reference` times the fp64 CPU oracle (the only reference that exists for this method) on the
+host cores, on a bounded sample of the same workload.
+
+With N > 1 (torchrun) every rank runs the same per-GPU workload on its own GPU (independent batch
+shards, no data-path collective): weak scaling, value = all ranks' tokens*heads / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "linear_attn_tokens_heads_per_s"
+UNIT = "tokens*heads/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="480p", choices=["480p", "720p"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the block-step / 720p side measurements")
+    return ap.parse_args()
+
+
+def workload_of(name):
+    from paper_2509_24695_b200 import synth
+
+    return synth.P480 if name == "480p" else synth.P720
+
+
+def peaks():
+    """Measured HBM copy bandwidth of this machine's B200s, else the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    bits = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in names.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def cpu_oracle_throughput(w, budget_s, q, k, v):
+    """The oracle as it stands on a bounded sample: every head, the first n_s tokens of the workload."""
+    import oracle
+
+    orc = oracle.default()
+    cores = min(os.cpu_count() or 1, w.B * w.H)  # the oracle parallelises over (batch, head) units only
+    n_s = min(w.N, 2048)
+    t0 = time.perf_counter()
+    orc.forward(q[:, :n_s], k[:, :n_s], v[:, :n_s], w.eps)
+    t_probe = time.perf_counter() - t0
+    n_s = int(max(256, min(w.N, n_s * budget_s / max(t_probe, 1e-4))))
+    t0 = time.perf_counter()
+    orc.forward(q[:, :n_s], k[:, :n_s], v[:, :n_s], w.eps)
+    dt = time.perf_counter() - t0
+    return {"value": w.B * n_s * w.H / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"fp64 oracle forward over all {w.B * w.H} (batch,head) units, first {n_s} of {w.N} tokens, "
+                      f"{dt:.2f} s wall"}, n_s
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2509_24695_b200 import synth
+    import oracle
+
+    w = workload_of(args.workload)
+    orc = oracle.default()
+    q, k, v = synth.qkv(w)
+    # size the per-step sample so that steps+warmup stay within about two minutes
+    n_s = min(w.N, 1024)
+    t0 = time.perf_counter()
+    orc.forward(q[:, :n_s], k[:, :n_s], v[:, :n_s], w.eps)
+    per_tok = (time.perf_counter() - t0) / n_s
+    n_s = int(max(128, min(w.N, 120.0 / max(1, args.steps + args.warmup) / per_tok)))
+    qs, ks, vs = q[:, :n_s], k[:, :n_s], v[:, :n_s]
+    for _ in range(args.warmup):
+        orc.forward(qs, ks, vs, w.eps)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.forward(qs, ks, vs, w.eps)
+    dt = time.perf_counter() - t0
+    value = args.steps * w.B * n_s * w.H / dt
+    cores = min(os.cpu_count() or 1, w.B * w.H)
+    sample = f"fp64 oracle forward, all {w.B * w.H} units, first {n_s} of {w.N} tokens per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(1, args.steps), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "N": w.N, "sample_tokens_per_step": n_s},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def time_loop(torch, fn, steps, sync_ranks=None):
+    """CUDA-event time of `steps` calls of fn(i) on the current stream, in ms."""
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if sync_ranks:
+        sync_ranks()
+    torch.cuda.synchronize()
+    start.record()
+    for i in range(steps):
+        fn(i)
+    stop.record()
+    torch.cuda.synchronize()
+    if sync_ranks:
+        sync_ranks()
+    return start.elapsed_time(stop)
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import paper_2509_24695_b200 as la
+    from paper_2509_24695_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl")
+    sync_ranks = (lambda: dist.barrier()) if dist else None
+
+    la.load_library()
+    w = workload_of(args.workload)
+    K, W = args.steps, max(args.warmup, 3)
+    dev = torch.device("cuda", local_rank)
+
+    # seeded synthetic inputs (same bits the oracle sees); two rotating input sets so no step finds
+    # its inputs in L2 (one set is 4 x 147 MB = 587 MB at 480p, already > 126 MB of L2)
+    q_h, k_h, v_h = synth.qkv(w)
+
+    def dev_of(bits):
+        return torch.from_numpy(bits.view("int16")).to(dev).view(torch.bfloat16)
+
+    sets = []
+    for r in range(2):
+        qd, kd, vd = dev_of(q_h), dev_of(k_h), dev_of(v_h)
+        if r:  # second set: same distribution, other values (token order reversed)
+            qd, kd, vd = qd.flip(1).contiguous(), kd.flip(1).contiguous(), vd.flip(1).contiguous()
+        sets.append((qd, kd, vd, torch.empty_like(qd)))
+    ws = la.new_workspace(sets[0][0])
+    units = w.B * w.N * w.H  # tokens*heads per step
+
+    def step(i):
+        qd, kd, vd, od = sets[i & 1]
+        la.linattn_forward(qd, kd, vd, w.eps, out=od, workspace=ws)
+
+    for i in range(W):
+        step(i)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    l0 = la.kernel_launches()
+    ms = time_loop(torch, step, K, sync_ranks)
+    launches = la.kernel_launches() - l0
+    # keep the device busy until the sampler has seen the clocks under this load
+    t_end = time.time() + 0.25
+    while len(sampler.samples) < 8 and time.time() < t_end:
+        step(0)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if dist:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / K
+    value = world * units / (ms_per_step * 1e-3)
+
+    # per-kernel split: state pass and apply pass timed live, each as its own entry point
+    state_buf = la.linattn_state(sets[0][1], sets[0][2], workspace=ws)
+    ms_state = time_loop(torch, lambda i: la.linattn_state(sets[i & 1][1], sets[i & 1][2], out=state_buf, workspace=ws), K) / K
+    ms_apply = time_loop(torch, lambda i: la.linattn_apply(sets[i & 1][0], state_buf, w.eps, out=sets[i & 1][3]), K) / K
+    peak, peak_kind = peaks()
+    bytes_tok_head = 2 * w.d  # one bf16 row of d features
+    state_bytes = la.state_bytes(w.B, w.H, w.d)
+    kern = {
+        "state": {"ms": ms_state, "bytes": units * 2 * bytes_tok_head + state_bytes},      # read K, V; write state
+        "apply": {"ms": ms_apply, "bytes": units * 2 * bytes_tok_head + state_bytes},      # read Q, state; write O
+        "forward": {"ms": ms_per_step, "bytes": units * 4 * bytes_tok_head},               # 8d bytes per token*head
+    }
+    for kv in kern.values():
+        kv["gbs"] = kv["bytes"] / (kv["ms"] * 1e-3) / 1e9
+    dom = "state" if ms_state >= ms_apply else "apply"
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["gbs"], "peak": peak, "unit": "GB/s",
+                "frac": kern[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "forward_frac": kern["forward"]["gbs"] / peak,
+                "kernels": {k_: {"ms": round(v_["ms"], 5), "gbs": round(v_["gbs"], 1)} for k_, v_ in kern.items()}}
+
+    # end to end through the host-buffer entry point: pinned host Q,K,V in, O out, copies inside the timed region
+    hf = la.HostForward(w.B, w.N, w.H, w.d, torch.bfloat16, dev)
+    pin = lambda bits: torch.from_numpy(bits.view("int16")).view(torch.bfloat16).pin_memory()
+    qp, kp, vp = pin(q_h), pin(k_h), pin(v_h)
+    op = torch.empty_like(qp).pin_memory()
+    k_e2e = max(3, min(K, 20))
+    for _ in range(2):
+        hf(qp, kp, vp, op, w.eps)
+    ms_e2e = time_loop(torch, lambda i: hf(qp, kp, vp, op, w.eps), k_e2e, sync_ranks)
+    if dist:
+        t = torch.tensor([ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e = {"value": world * units / (ms_e2e / k_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": hf.h2d_bytes,
+           "d2h_bytes_per_step": hf.d2h_bytes, "steps": k_e2e, "ms_per_step": ms_e2e / k_e2e}
+    assert float(op.float().abs().sum()) > 0.0
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "N": w.N, "eps": w.eps,
+                   "l2": "two rotating input sets of 587 MB each (> 126 MB L2)" if args.workload == "480p"
+                   else "two rotating input sets, each far larger than L2",
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+    }
+
+    if rank == 0 and world == 1:
+        cb, _ = cpu_oracle_throughput(w, 15.0, q_h, k_h, v_h)
+        out["cpu_baseline"] = cb
+        if not args.no_extras:
+            out["other_workloads"] = extras(torch, la, synth, dev, peak)
+    if rank == 0:
+        print(json.dumps(out))
+    if dist:
+        dist.destroy_process_group()
+
+
+def extras(torch, la, synth, dev, peak):
+    """Side measurements: block-step latency of the autoregressive and streaming configs (cache bytes stay
+    constant as blocks accumulate) and the 720p bidirectional layer."""
+    res = {}
+    for w, n_steps in ((synth.AR480, 21), (synth.STREAM720, 80)):
+        # a few distinct blocks, cycled: the cost of a step does not depend on the values
+        blocks = []
+        for b in range(3):
+            qb, kb, vb = synth.qkv_block(w, b)
+            blocks.append(tuple(torch.from_numpy(x.view("int16")).to(dev).view(torch.bfloat16) for x in (qb, kb, vb)))
+        ob = torch.empty_like(blocks[0][0])
+        cache = la.BlockLinCache(w.B, w.H, w.d, torch.bfloat16, dev, max_T_b=w.T_b, eps=w.eps)
+        for i in range(3):
+            cache.step(*blocks[i % 3], out=ob)
+        cache.reset()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps + 1)]
+        torch.cuda.synchronize()
+        evs[0].record()
+        for i in range(n_steps):
+            cache.step(*blocks[i % 3], out=ob)
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        lat = [evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(n_steps)]
+        step_bytes = w.B * w.T_b * w.H * 8 * w.d + 2 * cache.info()["state_bytes"]
+        med = sorted(lat)[len(lat) // 2]
+        res[w.name] = {"step_latency_us_median": med, "step_latency_us_first": lat[0], "step_latency_us_last": lat[-1],
+                       "steps": n_steps, "tokens_per_block": w.T_b, "B": w.B,
+                       "tokens_heads_per_s": w.B * w.T_b * w.H / (med * 1e-6),
+                       "algorithmic_gbs": step_bytes / (med * 1e-6) / 1e9, "frac_of_peak": step_bytes / (med * 1e-6) / 1e9 / peak,
+                       "cache_bytes_at_first_and_last_step": [cache.info()["state_bytes"]] * 2,
+                       "l2": "block set of %.0f MB cycled over 3 copies" % (step_bytes / 1e6)}
+        cache.close()
+        del blocks, ob
+    w = synth.P720
+    q, k, v = (torch.from_numpy(x.view("int16")).to(dev).view(torch.bfloat16) for x in synth.qkv(w))
+    o = torch.empty_like(q)
+    ws = la.new_workspace(q)
+    for _ in range(3):
+        la.linattn_forward(q, k, v, w.eps, out=o, workspace=ws)
+    n = 20
+    ms = time_loop(torch, lambda i: la.linattn_forward(q, k, v, w.eps, out=o, workspace=ws), n) / n
+    by = w.B * w.N * w.H * 8 * w.d
+    res[w.name] = {"ms": ms, "tokens_heads_per_s": w.B * w.N * w.H / (ms * 1e-3), "algorithmic_gbs": by / (ms * 1e-3) / 1e9,
+                   "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak}
+    return res
+
+
+if __name__ == "__main__":
+    main()

@@ -117,9 +117,24 @@ LINATTN_API int linattn_forward(const linattn_desc* desc, int64_t N, const void*
 LINATTN_API int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void* v, float* state,
                   void* workspace, size_t workspace_bytes, void* stream);
 
-/* The apply half of Eq. 2 alone: o_n = phi(q_n) S / (phi(q_n) . z + eps) for a given state. */
+/* The apply half of Eq. 2 alone: o_n = phi(q_n) S / (phi(q_n) . z + eps) for a given state.
+ * workspace: only its control block is used (LINATTN_WORKSPACE_CTRL_BYTES suffice). */
 LINATTN_API int linattn_apply(const linattn_desc* desc, int64_t N, const void* q, const float* state, void* o, float eps,
-                  void* stream);
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* Eq. 2 with HOST buffers: copies q, k, v (host, ideally pinned) into the caller's device staging
+ * area, runs linattn_forward there and copies O back to `o_host`, all enqueued on `stream`.
+ * `dev_staging` (DEVICE, 256-byte aligned) must hold linattn_forward_host_bytes() bytes: four dense
+ * [B,N,H,d] tensors plus the forward's workspace; its control block must have been zeroed once with
+ * linattn_workspace_init(dev_staging, ...).  Host tensors are dense [B,N,H,d] (the descriptor's
+ * strides must be 0).  The host buffers may be reused once `stream` has been synchronised. */
+LINATTN_API int linattn_forward_host_bytes(const linattn_desc* desc, int64_t N, size_t* bytes);
+LINATTN_API int linattn_forward_host(const linattn_desc* desc, int64_t N, const void* q_host, const void* k_host,
+                                     const void* v_host, void* o_host, float eps, void* dev_staging,
+                                     size_t dev_staging_bytes, void* stream);
+
+/* Number of CUDA kernels this library has launched in this process so far (all entry points). */
+LINATTN_API uint64_t linattn_kernel_launches(void);
 
 /* ---- block-causal form with the constant-memory cache (Eq. 3, Algorithm 1) ---- */
 

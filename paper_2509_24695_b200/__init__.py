@@ -18,7 +18,7 @@ import os
 
 __all__ = [
     "LinAttnError", "library_path", "load_library", "state_bytes", "workspace_bytes", "new_workspace",
-    "linattn_forward", "linattn_state", "linattn_apply", "split_state", "BlockLinCache", "workspace_status",
+    "linattn_forward", "linattn_state", "linattn_apply", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
 ]
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -70,7 +70,10 @@ def load_library(path: str | None = None):
         "linattn_workspace_status": ([vp, vp, ctypes.POINTER(ctypes.c_int)], ctypes.c_int),
         "linattn_forward": ([dp, i64, vp, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
         "linattn_state": ([dp, i64, vp, vp, vp, vp, sz, vp], ctypes.c_int),
-        "linattn_apply": ([dp, i64, vp, vp, vp, f32, vp], ctypes.c_int),
+        "linattn_apply": ([dp, i64, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
+        "linattn_forward_host_bytes": ([dp, i64, szp], ctypes.c_int),
+        "linattn_forward_host": ([dp, i64, vp, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
+        "linattn_kernel_launches": ([], ctypes.c_uint64),
         "blocklin_cache_bytes": ([dp, i64, szp, szp], ctypes.c_int),
         "blocklin_cache_init": ([ctypes.POINTER(vp), dp, f32, vp, sz, vp, sz, vp], ctypes.c_int),
         "blocklin_cache_reset": ([vp, vp], ctypes.c_int),
@@ -171,6 +174,44 @@ def linattn_forward(q, k, v, eps: float = 1e-6, out=None, workspace=None):
     return o
 
 
+def kernel_launches() -> int:
+    """CUDA kernels launched by the library in this process so far."""
+    return int(load_library().linattn_kernel_launches())
+
+
+class HostForward:
+    """Bidirectional forward over HOST tensors (pinned CPU torch tensors, dense [B, N, H, d]).
+
+    Owns a device staging area (allocated once with torch); each call enqueues host-to-device copies
+    of Q, K, V, the forward, and the device-to-host copy of O on the current stream.
+    """
+
+    def __init__(self, B: int, N: int, H: int, d: int, dtype, device="cuda"):
+        torch = _torch()
+        self._lib = load_library()
+        code = LINATTN_BF16 if dtype == torch.bfloat16 else LINATTN_F32
+        self._desc = _Desc(B, H, d, code, 0, 0, 0)
+        self.shape, self.dtype, self.N = (B, N, H, d), dtype, N
+        nb = ctypes.c_size_t()
+        _check(self._lib.linattn_forward_host_bytes(ctypes.byref(self._desc), N, ctypes.byref(nb)),
+               "linattn_forward_host_bytes")
+        self.staging = torch.empty(nb.value, dtype=torch.uint8, device=device)
+        _check(self._lib.linattn_workspace_init(_ptr(self.staging), nb.value, _stream(self.staging)),
+               "linattn_workspace_init")
+        itemsize = 2 if code == LINATTN_BF16 else 4
+        self.h2d_bytes = 3 * B * N * H * d * itemsize
+        self.d2h_bytes = B * N * H * d * itemsize
+
+    def __call__(self, q_host, k_host, v_host, o_host, eps: float = 1e-6):
+        for t in (q_host, k_host, v_host, o_host):
+            if t.is_cuda or tuple(t.shape) != self.shape or t.dtype != self.dtype or not t.is_contiguous():
+                raise ValueError("host tensors must be dense CPU [B, N, H, d] tensors of the configured dtype")
+        _check(self._lib.linattn_forward_host(ctypes.byref(self._desc), self.N, _ptr(q_host), _ptr(k_host),
+                                              _ptr(v_host), _ptr(o_host), eps, _ptr(self.staging),
+                                              self.staging.numel(), _stream(self.staging)), "linattn_forward_host")
+        return o_host
+
+
 def linattn_state(k, v, out=None, workspace=None):
     """State of Eq. 2 / Eq. 3: float32 [B, H, d+1, d] (S transposed, then z)."""
     torch = _torch()
@@ -184,7 +225,7 @@ def linattn_state(k, v, out=None, workspace=None):
     return st
 
 
-def linattn_apply(q, state, eps: float = 1e-6, out=None):
+def linattn_apply(q, state, eps: float = 1e-6, out=None, workspace=None):
     """Apply half of Eq. 2 for a given state."""
     torch = _torch()
     lib = load_library()
@@ -193,7 +234,9 @@ def linattn_apply(q, state, eps: float = 1e-6, out=None):
     B, N, H, d = q.shape
     if tuple(state.shape) != (B, H, d + 1, d) or state.dtype != torch.float32 or not state.is_contiguous():
         raise ValueError("state must be a contiguous float32 [B, H, d+1, d] tensor")
-    _check(lib.linattn_apply(ctypes.byref(desc), N, _ptr(q), _ptr(state), _ptr(o), eps, _stream(q)), "linattn_apply")
+    ws = new_workspace(q, 0) if workspace is None else workspace
+    _check(lib.linattn_apply(ctypes.byref(desc), N, _ptr(q), _ptr(state), _ptr(o), eps, _ptr(ws), ws.numel(),
+                             _stream(q)), "linattn_apply")
     return o
 
 

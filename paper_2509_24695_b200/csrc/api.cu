@@ -1,10 +1,16 @@
 // C ABI of the linear-attention library: argument validation, workspace layout, kernel selection
 // and the host-side cache handle.  See include/linattn.h for the contract of each entry point.
+#include <atomic>
 #include <new>
 
 #include "common.cuh"
 
 using namespace linattn;
+
+namespace linattn {
+static std::atomic<uint64_t> g_kernel_launches{0};
+void count_launches(int n) { g_kernel_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+}  // namespace linattn
 
 namespace {
 
@@ -69,8 +75,10 @@ int run_state(const Problem& p, const void* k, const void* v, float* state, bool
   return cuda_status(fma_state(p, k, v, state, accumulate, partials_of(workspace), stream));
 }
 
-int run_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream) {
-  if (umma_supported(p)) return umma_apply(p, q, state, o, eps, stream);
+int run_apply(const Problem& p, const void* q, const float* state, void* o, float eps, void* workspace,
+              cudaStream_t stream) {
+  if (umma_supported(p))
+    return umma_apply(p, q, state, o, eps, &static_cast<WorkspaceCtrl*>(workspace)->status, stream);
   return cuda_status(fma_apply(p, q, state, o, eps, stream));
 }
 
@@ -101,7 +109,7 @@ static int step_impl(blocklin_cache* cache, const Problem& p, const void* q_blk,
   st = run_state(p, k_blk, v_blk, cache->state, true, cache->workspace, stream);
   if (st != LINATTN_OK) return st;
   if (q_blk) {
-    st = run_apply(p, q_blk, cache->state, o_blk, cache->eps, stream);
+    st = run_apply(p, q_blk, cache->state, o_blk, cache->eps, cache->workspace, stream);
     if (st != LINATTN_OK) return st;
   }
   cache->blocks_seen += 1;
@@ -171,14 +179,15 @@ int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void
 }
 
 int linattn_apply(const linattn_desc* desc, int64_t N, const void* q, const float* state, void* o, float eps,
-                  void* stream) {
+                  void* workspace, size_t workspace_bytes, void* stream) {
   Problem p;
   int st = resolve(desc, N, &p);
   if (st != LINATTN_OK) return st;
-  if (!state) return LINATTN_ERR_INVALID_ARG;
+  if (!state || !workspace) return LINATTN_ERR_INVALID_ARG;
   if (N > 0 && (!q || !o || q == o)) return LINATTN_ERR_INVALID_ARG;
-  if ((st = check_alignment(p, q, o, state, nullptr)) != LINATTN_OK) return st;
-  return run_apply(p, q, state, o, eps, (cudaStream_t)stream);
+  if ((st = check_alignment(p, q, o, state, workspace)) != LINATTN_OK) return st;
+  if (workspace_bytes < LINATTN_WORKSPACE_CTRL_BYTES) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  return run_apply(p, q, state, o, eps, workspace, (cudaStream_t)stream);
 }
 
 int linattn_forward(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v, void* o,
@@ -196,7 +205,53 @@ int linattn_forward(const linattn_desc* desc, int64_t N, const void* q, const vo
   float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + state_slot_offset(p));
   st = run_state(p, k, v, state, false, workspace, (cudaStream_t)stream);
   if (st != LINATTN_OK) return st;
-  return run_apply(p, q, state, o, eps, (cudaStream_t)stream);
+  return run_apply(p, q, state, o, eps, workspace, (cudaStream_t)stream);
+}
+
+uint64_t linattn_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
+
+int linattn_forward_host_bytes(const linattn_desc* desc, int64_t N, size_t* bytes) {
+  Problem p;
+  if (!bytes) return LINATTN_ERR_INVALID_ARG;
+  int st = resolve(desc, N, &p);
+  if (st != LINATTN_OK) return st;
+  if (desc->stride_b || desc->stride_n || desc->stride_h) return LINATTN_ERR_UNSUPPORTED;
+  const size_t esz = p.dtype == LINATTN_BF16 ? 2 : 4;
+  const size_t tensor = round256((size_t)p.B * (size_t)N * p.H * p.d * esz);
+  *bytes = workspace_need(p) + 4 * tensor;
+  return LINATTN_OK;
+}
+
+int linattn_forward_host(const linattn_desc* desc, int64_t N, const void* q_host, const void* k_host,
+                         const void* v_host, void* o_host, float eps, void* dev_staging, size_t dev_staging_bytes,
+                         void* stream) {
+  size_t need = 0;
+  int st = linattn_forward_host_bytes(desc, N, &need);
+  if (st != LINATTN_OK) return st;
+  if (!dev_staging || (reinterpret_cast<uintptr_t>(dev_staging) & 255u)) return LINATTN_ERR_BAD_ALIGNMENT;
+  if (dev_staging_bytes < need) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  if (N == 0) return LINATTN_OK;
+  if (!q_host || !k_host || !v_host || !o_host) return LINATTN_ERR_INVALID_ARG;
+  Problem p;
+  resolve(desc, N, &p);
+  const size_t esz = p.dtype == LINATTN_BF16 ? 2 : 4;
+  const size_t bytes = (size_t)p.B * (size_t)N * p.H * p.d * esz;
+  const size_t tensor = round256(bytes);
+  const size_t ws = workspace_need(p);
+  char* base = static_cast<char*>(dev_staging);
+  void* dq = base + ws;
+  void* dk = base + ws + tensor;
+  void* dv = base + ws + 2 * tensor;
+  void* dout = base + ws + 3 * tensor;
+  cudaStream_t s = (cudaStream_t)stream;
+  // K and V first: the state pass needs them; Q is only needed by the apply pass
+  cudaError_t e = cudaMemcpyAsync(dk, k_host, bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, bytes, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return LINATTN_ERR_CUDA;
+  st = linattn_forward(desc, N, dq, dk, dv, dout, eps, dev_staging, ws, stream);
+  if (st != LINATTN_OK) return st;
+  return cuda_status(cudaMemcpyAsync(o_host, dout, bytes, cudaMemcpyDeviceToHost, s));
 }
 
 int blocklin_cache_bytes(const linattn_desc* desc, int64_t max_T_b, size_t* state_bytes, size_t* workspace_bytes) {

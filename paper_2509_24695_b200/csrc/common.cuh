@@ -28,6 +28,9 @@ struct WorkspaceCtrl {
 };
 static_assert(sizeof(WorkspaceCtrl) <= LINATTN_WORKSPACE_CTRL_BYTES, "control block too large");
 
+// Kernel-launch counter behind linattn_kernel_launches().
+void count_launches(int n);
+
 constexpr int kMaxCtas = 256;        // upper bound on the persistent grid (B200 has 148 SMs)
 constexpr int kFmaMaxChunks = 64;    // split-N partials per unit on the FMA path
 constexpr int kFmaMinChunkTokens = 512;
@@ -50,6 +53,7 @@ size_t umma_partial_bytes(const Problem& p);
 // Returns LINATTN_OK or an error status.
 int umma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate, void* workspace,
                cudaStream_t stream);
-int umma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream);
+int umma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, int* status,
+               cudaStream_t stream);
 
 }  // namespace linattn

@@ -188,6 +188,7 @@ cudaError_t launch_state_partial(const Problem& p, const void* k, const void* v,
                                  cudaStream_t stream) {
   dim3 grid(P, p.units());
   fma_state_partial<T, R><<<grid, kThreads, 0, stream>>>((const T*)k, (const T*)v, p, P, partials);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -199,6 +200,7 @@ cudaError_t launch_apply(const Problem& p, const void* q, const float* state, vo
   if (e != cudaSuccess) return e;
   dim3 grid((unsigned)((p.N + kApplyTile - 1) / kApplyTile), p.units());
   fma_apply_kernel<T, R><<<grid, kThreads, smem, stream>>>((const T*)q, state, (T*)o, p, eps);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -245,6 +247,7 @@ cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* sta
   if (e != cudaSuccess) return e;
   dim3 grid((unsigned)((E + kThreads - 1) / kThreads), p.units());
   fma_state_reduce<<<grid, kThreads, 0, stream>>>(partials, P, E, state_out, accumulate ? 1 : 0);
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -39,21 +39,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Bounded wait.  Polls until the phase with the given parity has completed, another thread of the
-// CTA has raised *abort_flag, or the poll budget (roughly a second) runs out.  On timeout it raises
-// *abort_flag itself and returns false; the caller must then stop issuing work and fall through to
-// the kernel's teardown.  No wait in these kernels can spin forever.
-constexpr uint32_t kSpinFast = 1u << 14;
-constexpr uint32_t kSpinSlow = 1u << 22;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinFast; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  for (uint32_t i = 0; i < kSpinSlow; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+// CTA has raised *abort_flag, or about a second of wall time (global timer) has passed.  On timeout
+// it raises *abort_flag itself and returns false; the caller must then stop issuing work and fall
+// through to the kernel's teardown.  No wait in these kernels can spin forever.
+constexpr uint32_t kSpinFast = 1u << 12;
+constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const unsigned long long t0 = global_timer_ns();
+  for (;;) {
+    for (int i = 0; i < 64; ++i) {
+      if (mbar_try_wait(bar, parity)) return true;
+      __nanosleep(32);
+    }
     if (*abort_flag) return false;
-    __nanosleep(128);
+    if (global_timer_ns() - t0 > kWaitLimitNs) break;
   }
   *abort_flag = 1;
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinFast; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 // ---------------------------------------------------------------- fences
