@@ -38,6 +38,9 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="480p", choices=["480p", "720p"])
     ap.add_argument("--no-extras", action="store_true", help="skip the block-step / 720p side measurements")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="time the device kernels only (no host-buffer leg, no CPU oracle, no side measurements): "
+                         "the short command used under a profiler")
     return ap.parse_args()
 
 
@@ -272,22 +275,24 @@ def main():
                 "forward_frac": kern["forward"]["gbs"] / peak,
                 "kernels": {k_: {"ms": round(v_["ms"], 5), "gbs": round(v_["gbs"], 1)} for k_, v_ in kern.items()}}
 
-    # end to end through the host-buffer entry point: pinned host Q,K,V in, O out, copies inside the timed region
-    hf = la.HostForward(w.B, w.N, w.H, w.d, torch.bfloat16, dev)
-    pin = lambda bits: torch.from_numpy(bits.view("int16")).view(torch.bfloat16).pin_memory()
-    qp, kp, vp = pin(q_h), pin(k_h), pin(v_h)
-    op = torch.empty_like(qp).pin_memory()
-    k_e2e = max(3, min(K, 20))
-    for _ in range(2):
-        hf(qp, kp, vp, op, w.eps)
-    ms_e2e = time_loop(torch, lambda i: hf(qp, kp, vp, op, w.eps), k_e2e, sync_ranks)
-    if dist:
-        t = torch.tensor([ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e = {"value": world * units / (ms_e2e / k_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": hf.h2d_bytes,
-           "d2h_bytes_per_step": hf.d2h_bytes, "steps": k_e2e, "ms_per_step": ms_e2e / k_e2e}
-    assert float(op.float().abs().sum()) > 0.0
+    e2e = None
+    if not args.kernels_only:
+        # end to end through the host-buffer entry point: pinned host Q,K,V in, O out, copies inside the timed region
+        hf = la.HostForward(w.B, w.N, w.H, w.d, torch.bfloat16, dev)
+        pin = lambda bits: torch.from_numpy(bits.view("int16")).view(torch.bfloat16).pin_memory()
+        qp, kp, vp = pin(q_h), pin(k_h), pin(v_h)
+        op = torch.empty_like(qp).pin_memory()
+        k_e2e = max(3, min(K, 20))
+        for _ in range(2):
+            hf(qp, kp, vp, op, w.eps)
+        ms_e2e = time_loop(torch, lambda i: hf(qp, kp, vp, op, w.eps), k_e2e, sync_ranks)
+        if dist:
+            t = torch.tensor([ms_e2e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": world * units / (ms_e2e / k_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": hf.h2d_bytes,
+               "d2h_bytes_per_step": hf.d2h_bytes, "steps": k_e2e, "ms_per_step": ms_e2e / k_e2e}
+        assert float(op.float().abs().sum()) > 0.0
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -300,7 +305,7 @@ def main():
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
     }
 
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.kernels_only:
         cb, _ = cpu_oracle_throughput(w, 15.0, q_h, k_h, v_h)
         out["cpu_baseline"] = cb
         if not args.no_extras:

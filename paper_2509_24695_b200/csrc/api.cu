@@ -68,18 +68,20 @@ inline float* partials_of(void* workspace) {
 
 int cuda_status(cudaError_t e) { return e == cudaSuccess ? LINATTN_OK : LINATTN_ERR_CUDA; }
 
-// state_out = (accumulate ? state_out : 0) + state(k, v)
-int run_state(const Problem& p, const void* k, const void* v, float* state, bool accumulate, void* workspace,
-              cudaStream_t stream) {
-  if (umma_supported(p)) return umma_state(p, k, v, state, accumulate, workspace, stream);
-  return cuda_status(fma_state(p, k, v, state, accumulate, partials_of(workspace), stream));
-}
-
-int run_apply(const Problem& p, const void* q, const float* state, void* o, float eps, void* workspace,
-              cudaStream_t stream) {
-  if (umma_supported(p))
-    return umma_apply(p, q, state, o, eps, &static_cast<WorkspaceCtrl*>(workspace)->status, stream);
-  return cuda_status(fma_apply(p, q, state, o, eps, stream));
+// state_out = (accumulate ? state_out : 0) + state(k, v), then (q non-null) o = apply(q, state_out).
+// On the tensor-core path both halves run in one launch.
+int run_passes(const Problem& p, const void* k, const void* v, const void* q, void* o, float* state, bool accumulate,
+               float eps, void* workspace, cudaStream_t stream) {
+  if (umma_supported(p)) {
+    UmmaCall c{k, v, q, o, state, accumulate, eps};
+    return umma_run(p, c, workspace, stream);
+  }
+  if (k) {
+    int st = cuda_status(fma_state(p, k, v, state, accumulate, partials_of(workspace), stream));
+    if (st != LINATTN_OK) return st;
+  }
+  if (q) return cuda_status(fma_apply(p, q, state, o, eps, stream));
+  return LINATTN_OK;
 }
 
 }  // namespace
@@ -106,12 +108,8 @@ static int step_impl(blocklin_cache* cache, const Problem& p, const void* q_blk,
   if (st != LINATTN_OK) return st;
   if (cache->workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
   if (p.N == 0) return LINATTN_OK;
-  st = run_state(p, k_blk, v_blk, cache->state, true, cache->workspace, stream);
+  st = run_passes(p, k_blk, v_blk, q_blk, o_blk, cache->state, true, cache->eps, cache->workspace, stream);
   if (st != LINATTN_OK) return st;
-  if (q_blk) {
-    st = run_apply(p, q_blk, cache->state, o_blk, cache->eps, cache->workspace, stream);
-    if (st != LINATTN_OK) return st;
-  }
   cache->blocks_seen += 1;
   cache->tokens_seen += p.N;
   return LINATTN_OK;
@@ -175,7 +173,8 @@ int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void
   if (N > 0 && (!k || !v)) return LINATTN_ERR_INVALID_ARG;
   if ((st = check_alignment(p, k, v, state, workspace)) != LINATTN_OK) return st;
   if (workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
-  return run_state(p, k, v, state, false, workspace, (cudaStream_t)stream);
+  if (N == 0) return cuda_status(cudaMemsetAsync(state, 0, state_bytes_of(p), (cudaStream_t)stream));  // empty sum
+  return run_passes(p, k, v, nullptr, nullptr, state, false, 0.f, workspace, (cudaStream_t)stream);
 }
 
 int linattn_apply(const linattn_desc* desc, int64_t N, const void* q, const float* state, void* o, float eps,
@@ -187,7 +186,8 @@ int linattn_apply(const linattn_desc* desc, int64_t N, const void* q, const floa
   if (N > 0 && (!q || !o || q == o)) return LINATTN_ERR_INVALID_ARG;
   if ((st = check_alignment(p, q, o, state, workspace)) != LINATTN_OK) return st;
   if (workspace_bytes < LINATTN_WORKSPACE_CTRL_BYTES) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
-  return run_apply(p, q, state, o, eps, workspace, (cudaStream_t)stream);
+  if (N == 0) return LINATTN_OK;
+  return run_passes(p, nullptr, nullptr, q, o, const_cast<float*>(state), false, eps, workspace, (cudaStream_t)stream);
 }
 
 int linattn_forward(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v, void* o,
@@ -203,9 +203,7 @@ int linattn_forward(const linattn_desc* desc, int64_t N, const void* q, const vo
   if (N == 0) return LINATTN_OK;
   // the forward keeps its reduced state in the workspace, after the partials
   float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + state_slot_offset(p));
-  st = run_state(p, k, v, state, false, workspace, (cudaStream_t)stream);
-  if (st != LINATTN_OK) return st;
-  return run_apply(p, q, state, o, eps, workspace, (cudaStream_t)stream);
+  return run_passes(p, k, v, q, o, state, false, eps, workspace, (cudaStream_t)stream);
 }
 
 uint64_t linattn_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }

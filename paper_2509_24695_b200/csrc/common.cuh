@@ -47,13 +47,20 @@ cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* sta
                       float* partials, cudaStream_t stream);
 cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream);
 
-// ---- tensor-core (tcgen05 + TMA) kernels, bf16, d in {32, 64, 112, 128} ----
+// ---- tensor-core (tcgen05 + TMA) kernel, bf16, d in {64, 112, 128} ----
+// One launch runs the state pass (k, v non-null), the apply pass (q, o non-null), or both back to back.
+struct UmmaCall {
+  const void* k;
+  const void* v;
+  const void* q;
+  void* o;
+  float* state;     // written by the state pass (on top of its contents when `accumulate`), read by the apply pass
+  bool accumulate;
+  float eps;
+};
 bool umma_supported(const Problem& p);
 size_t umma_partial_bytes(const Problem& p);
 // Returns LINATTN_OK or an error status.
-int umma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate, void* workspace,
-               cudaStream_t stream);
-int umma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, int* status,
-               cudaStream_t stream);
+int umma_run(const Problem& p, const UmmaCall& call, void* workspace, cudaStream_t stream);
 
 }  // namespace linattn

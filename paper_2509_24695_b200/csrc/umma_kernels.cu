@@ -1,31 +1,35 @@
-// Tensor-core kernels for bf16 ReLU linear attention on sm_100a: TMA tiles into shared memory,
-// a ReLU pass in place, tcgen05.mma with fp32 accumulators in tensor memory, results streamed out.
+// Tensor-core kernel for bf16 ReLU linear attention on sm_100a: TMA tiles into shared memory, a ReLU
+// pass in place, tcgen05.mma with fp32 accumulators in tensor memory, results streamed out.
 //
-// Both contractions of the method are dense and run on the tensor cores, but the kernels are
-// HBM-bound (about d/2 FLOP per byte); everything here is organised around keeping TMA loads in
-// flight on every SM.
+// Both contractions of the method are dense and run on the tensor cores, but the work is HBM-bound
+// (about d/2 FLOP per byte); everything here is organised around keeping TMA loads in flight on every SM.
 //
-//   umma_state_kernel   S = sum_n phi(k_n)^T v_n and z = sum_n phi(k_n)   (Eq. 2 / Eq. 3 state).
-//                       A = phi(K)^T and B = [V | 1] are both token-major in memory, i.e. MN-major
-//                       UMMA operands; the contraction index is the token.  The extra "ones" column
-//                       makes z fall out of the same MMA as column 128 of the accumulator.
-//                       Work is split over tokens across the grid (split-N); every CTA writes one
-//                       fp32 partial per (head group) segment it covered.
-//   umma_reduce_kernel  sums the partials of each head in a fixed order (deterministic), optionally
-//                       on top of the existing state: the cache update of Eq. 3.
-//   umma_apply_kernel   o_n = phi(q_n) S / (phi(q_n).z + eps).  A = phi(Q) tile (K-major), B = S
-//                       split into bf16 hi + lo parts (two MMAs per K step, so S keeps ~16 mantissa
-//                       bits), with z as an extra row of B so the denominator is one more
-//                       accumulator column.  The epilogue divides, rounds to bf16 and TMA-stores.
+// ONE persistent, cooperatively launched kernel runs up to three passes back to back:
 //
-// Head dims 32 and 64 pack 4 / 2 heads into one 128-feature operand (the cross-head blocks of the
-// product are ignored / zero); 112 pads to 128 through TMA out-of-bounds zero fill.
+//   state pass   S = sum_n phi(k_n)^T v_n and z = sum_n phi(k_n)   (Eq. 2 / Eq. 3 state).
+//                A = phi(K)^T and B = [V | 1] are both token-major in memory, i.e. MN-major UMMA
+//                operands; the contraction index is the token.  The "ones" column makes z fall out of
+//                the same MMA as one more accumulator column.  Work is split over tokens across the
+//                grid (split-N); every CTA writes one fp32 partial record per unit segment it covered.
+//   reduce       after a grid barrier every CTA sums a slice of the state over the partial records in
+//                a fixed order (deterministic), optionally on top of the existing state: the cache
+//                update of Eq. 3.  A second grid barrier publishes the state.
+//   apply pass   o_n = phi(q_n) S / (phi(q_n).z + eps).  A = phi(Q) tile (K-major), B = S split into
+//                bf16 hi + lo parts (two MMAs per K step, so S keeps ~16 mantissa bits), with z as an
+//                extra row of B so the denominator is one more accumulator column.  The epilogue
+//                divides, rounds to bf16 and a dedicated warp TMA-stores the tile.
 //
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 ReLU
-// pass, warps 6-9 epilogue.  All cross-role synchronisation is by mbarriers with bounded waits; a
-// wait that runs out raises a CTA-wide abort flag, records LINATTN_ERR_TIMEOUT in the workspace
-// status word, and every role falls through to the common teardown (TMEM is freed, loads in flight
-// are waited for with a bound).
+// The first Q tiles of the apply pass are fetched before the grid barriers (Q does not depend on the
+// state), so HBM stays busy while the partials are reduced.
+//
+// Head dim 64 packs two heads into one 128-feature operand (the cross-head blocks of the product are
+// ignored / zero); 112 pads to 128 through TMA out-of-bounds zero fill.
+//
+// Warp roles (352 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 ReLU
+// pass, warps 6-9 epilogue, warp 10 output stores.  All cross-role synchronisation is by mbarriers
+// with bounded waits, and the grid barrier is bounded too; a wait that runs out raises a CTA-wide
+// abort flag, records LINATTN_ERR_TIMEOUT in the workspace status word, and every role falls through
+// to the common teardown (TMEM is freed, loads in flight are waited for with a bound).
 #include <cuda.h>
 
 #include "common.cuh"
@@ -36,54 +40,128 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kReluThread0 = 64;    // warps 2-5
 constexpr int kEpiThread0 = 192;    // warps 6-9
+constexpr int kStoreWarp = 10;
 constexpr int kTileApply = 128;     // tokens per apply tile (= UMMA M)
 constexpr int kTileState = 64;      // tokens per state stage (4 UMMA K steps of 16 tokens)
 constexpr int kRowBytes = 128;      // one swizzle row: 64 bf16
+constexpr int kBox = kTileState * kRowBytes;  // 8 KB: one 64-feature box of a state stage
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;     // TMEM columns between the two accumulator buffers
 
 template <int D>
 struct Cfg {
-  static constexpr int G = D == 32 ? 4 : D == 64 ? 2 : 1;   // heads packed into one 128-feature operand
+  static constexpr int G = D == 64 ? 2 : 1;                  // heads packed into one 128-feature operand
   static constexpr int FEAT = G * D;                         // 112 or 128 live features per group
   static constexpr int KSTEPS = FEAT / 16;                   // apply: K steps over features
   static constexpr int ZROW = D == 112 ? 112 : 128;          // apply: accumulator column of the first denominator
   static constexpr int NAPPLY = D == 112 ? 128 : 144;        // apply MMA N
-  static constexpr int NSTATE = 144;                         // state MMA N: 128 value columns + the ones chunk
-  static constexpr int BOX_D = D < 64 ? D : 64;              // TMA box: features ...
-  static constexpr int BOX_H = 64 / BOX_D;                   // ... x heads = 64 elements = one 128-byte row
+  // state: with D = 112 the 1 sits in value column 112 (zero padding the TMA wrote), else in a
+  // constant extra chunk of the stage
+  static constexpr bool ONES_BOX = D != 112;
+  static constexpr int NSTATE = ONES_BOX ? 144 : 128;        // state MMA N
+  static constexpr int ZCOL = ONES_BOX ? 128 : 112;          // state accumulator column that holds z
+  static constexpr int BOX_D = 64;                           // TMA box: features ...
+  static constexpr int BOX_H = 1;                            // ... x heads
   static constexpr int SBOX_BYTES = NAPPLY * kRowBytes;      // one 64-feature K box of the S operand
   static constexpr int S_BYTES = 4 * SBOX_BYTES;             // (hi, lo) x 2 K boxes
   static constexpr int APPLY_SLOTS = D == 112 ? 5 : 4;
-  static constexpr int APPLY_SLOT_BYTES = 2 * kTileApply * kRowBytes;  // 32 KB: two 64-feature boxes
-  static constexpr int STATE_STAGES = 5;
-  static constexpr int BOX_BYTES_STATE = kTileState * kRowBytes;       // 8 KB
-  static constexpr int STATE_STAGE_BYTES = 5 * BOX_BYTES_STATE;        // V0 V1 ONES K0 K1
-  static constexpr size_t APPLY_SMEM = 1024 + S_BYTES + APPLY_SLOTS * APPLY_SLOT_BYTES + 512;
-  static constexpr size_t STATE_SMEM = 1024 + STATE_STAGES * STATE_STAGE_BYTES + 512;
+  static constexpr int SLOT_BYTES = 2 * kTileApply * kRowBytes;        // 32 KB: two 64-feature boxes
+  static constexpr int STAGE_BYTES = (ONES_BOX ? 5 : 4) * kBox;        // V0 V1 [ONES] K0 K1
+  static constexpr int KOFF = (ONES_BOX ? 3 : 2) * kBox;               // K boxes within a stage
+  static constexpr int DATA_BYTES = S_BYTES + APPLY_SLOTS * SLOT_BYTES;
+  static constexpr int STATE_STAGES = DATA_BYTES / STAGE_BYTES;        // the state pass uses the whole data area
+  static constexpr int BAR_BYTES = 1024;
+  static constexpr size_t SMEM = 1024 + DATA_BYTES + BAR_BYTES;
 };
 
-struct UmmaParams {
+// How the (unit, token tile) work of one pass is dealt to the persistent grid.
+//
+// A unit is one (batch, head group); its tiles are consecutive token ranges.  With U units and `grid`
+// CTAs, the first P*U CTAs ("column" CTAs, P = grid / U) take tiles [c*Lc, (c+1)*Lc) of unit j % U with
+// c = j / U and Lc = ceil(U*tpu / grid); the remaining R CTAs split the tiles [P*Lc, tpu) of all units
+// evenly, unit after unit.  Column CTAs of neighbouring heads therefore walk the same token range at
+// the same time.  That matters for head dims whose rows are not whole 128-byte lines (112 features =
+// 224 bytes): a line shared by two heads comes from DRAM once if both heads ask for it while it is
+// still in L2, and twice if their CTAs reach it tens of microseconds apart.
+struct Sched {
+  int U, tpu, grid;
+  int P, Lc, R;
+  int m;  // tiles per unit left to the R trailing CTAs: tpu - min(P*Lc, tpu)
+};
+
+// One CTA's share: flat positions [f0, f1); position f is tile tile_base + f % mm of unit
+// unit_base + f / mm, and the partial record of that unit's segment is rec_base + f / mm.
+struct Work {
+  long long f0, f1;
+  int mm, tile_base, unit_base, rec_base;
+};
+
+__host__ __device__ inline Work work_of(const Sched& s, int j) {
+  Work w;
+  w.f0 = w.f1 = 0; w.mm = 1; w.tile_base = 0; w.unit_base = 0; w.rec_base = 0;
+  if (j >= s.grid) return w;
+  if (j < s.P * s.U) {
+    const int t0 = (j / s.U) * s.Lc;
+    const int t1 = t0 + s.Lc < s.tpu ? t0 + s.Lc : s.tpu;
+    w.f1 = t1 > t0 ? t1 - t0 : 0;
+    w.mm = 0x7fffffff; w.tile_base = t0; w.unit_base = j % s.U; w.rec_base = j;
+  } else {
+    const int r = j - s.P * s.U;
+    const long long tot = (long long)s.U * s.m;
+    w.f0 = r * tot / s.R; w.f1 = (r + 1) * tot / s.R;
+    w.mm = s.m > 0 ? s.m : 1; w.tile_base = s.P * s.Lc; w.rec_base = s.P * s.U + r;
+  }
+  return w;
+}
+
+inline Sched make_sched(int U, long long tpu, int max_ctas) {
+  Sched s;
+  const long long total = (long long)U * tpu;
+  s.U = U; s.tpu = (int)tpu;
+  s.grid = (int)(total < max_ctas ? total : max_ctas);
+  if (s.grid < 1) s.grid = 1;
+  s.P = s.grid / U;
+  s.Lc = (int)((total + s.grid - 1) / s.grid);
+  const long long covered = (long long)s.P * s.Lc;
+  s.m = covered >= tpu ? 0 : (int)(tpu - covered);
+  s.R = s.grid - s.P * U;
+  return s;
+}
+
+// Walks a Work range tile by tile.
+struct TileWalk {
+  const Work w;
+  long long f;
+  int uo, tp;
+  __device__ explicit TileWalk(const Work& w_) : w(w_), f(w_.f0), uo((int)(w_.f0 / w_.mm)), tp((int)(w_.f0 % w_.mm)) {}
+  __device__ bool done() const { return f >= w.f1; }
+  __device__ int unit() const { return w.unit_base + uo; }
+  __device__ int tile() const { return w.tile_base + tp; }
+  __device__ int record() const { return w.rec_base + uo; }
+  __device__ bool seg_first() const { return f == w.f0 || tp == 0; }
+  __device__ bool seg_last() const { return f + 1 == w.f1 || tp == w.mm - 1; }
+  __device__ void next() { ++f; if (++tp == w.mm) { tp = 0; ++uo; } }
+};
+
+struct FusedParams {
   int B, H, HG;            // HG: head groups per batch entry = ceil(H / G)
-  long long N;
-  int tiles_per_unit;      // token tiles per (batch, head group) unit
-  long long total_tiles;   // units * tiles_per_unit
-  const float* state_in;   // apply: [B][H][(d+1)][d]
-  float* partials;         // state: one record of G head-states per (CTA, unit) segment
+  Sched sa, sc;            // state pass (64-token stages) and apply pass (128-token tiles)
+  int do_state, do_apply;
+  int accumulate;          // reduce on top of the existing state
+  float* state;            // [B][H][(d+1)][d]
+  float* partials;         // one record of G head-states per (CTA, unit) segment of the state pass
   float eps;
-  int* status;             // workspace status word
+  WorkspaceCtrl* ctrl;
 };
 
 // TMA coordinates (feature, head) of 64-element box `box` (0/1) of head group hg
 template <int D>
 __device__ __forceinline__ void box_coords(int box, int hg, int& c0, int& c1) {
-  using C = Cfg<D>;
-  if (C::G == 1) { c0 = 64 * box; c1 = hg; }
-  else if (C::G == 2) { c0 = 0; c1 = 2 * hg + box; }
-  else { c0 = 0; c1 = 4 * hg + 2 * box; }
+  if (Cfg<D>::G == 1) { c0 = 64 * box; c1 = hg; }
+  else { c0 = 0; c1 = 2 * hg + box; }
 }
 
 __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
@@ -108,208 +186,81 @@ __device__ __forceinline__ void relu_pass(uint8_t* base, int nchunks, int chunks
   }
 }
 
-// ============================================================================ state kernel
-// grid: persistent, CTA j covers flat stage indices [j*W/G, (j+1)*W/G) over (unit, 64-token stage).
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
-umma_state_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, UmmaParams p) {
-  using C = Cfg<D>;
-  constexpr int NS = C::STATE_STAGES;
-  constexpr int BOX = C::BOX_BYTES_STATE;
-  constexpr int STAGE = C::STATE_STAGE_BYTES;
-  constexpr uint32_t IDESC = make_idesc_bf16(128, C::NSTATE, true, true);
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = align1024(smem_raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NS * STAGE);
-  uint64_t* full = bars;             // TMA landed
-  uint64_t* ready = bars + NS;       // ReLU pass done
-  uint64_t* empty = bars + 2 * NS;   // MMAs that read the stage are complete
-  uint64_t* tfull = bars + 3 * NS;   // [2] accumulator complete
-  uint64_t* tempty = tfull + 2;      // [2] accumulator drained by the epilogue
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tempty + 2);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+// ---------------------------------------------------------------- grid barrier
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long t_begin = (long long)blockIdx.x * p.total_tiles / gridDim.x;
-  const long long t_end = (long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x;
-  const int tpu = p.tiles_per_unit;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&ready[s], 128); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 128); }
-    *abort_flag = 0;
-    fence_mbar_init();
-    prefetch_tensormap(&map_k);
-    prefetch_tensormap(&map_v);
-  }
-  // the constant "ones" chunk of every stage: value columns 128..191 of B, of which column 128 is 1
-  for (int idx = threadIdx.x; idx < NS * (BOX / 16); idx += kThreads) {
-    const int s = idx / (BOX / 16), c = idx % (BOX / 16);
-    const int row = c >> 3, phys = c & 7;
-    uint4 val = make_uint4(0, 0, 0, 0);
-    if ((phys ^ (row & 7)) == 0) val.x = 0x3F80u;  // bf16 1.0 in element 0 of logical chunk 0
-    *reinterpret_cast<uint4*>(smem + s * STAGE + 2 * BOX + c * 16) = val;
-  }
-  fence_proxy_async_smem();
-  if (warp == 1) { tmem_alloc(tmem_holder, kTmemCols); tmem_relinquish(); }
+// All CTAs of the (cooperatively launched, hence co-resident) grid meet here.  Sense-reversing and
+// self-resetting: the last CTA to arrive zeroes the counter and bumps the generation word the others
+// poll.  The poll is bounded (about a second); on expiry the CTA raises its abort flag and goes on
+// to the teardown.
+__device__ __forceinline__ void grid_barrier(WorkspaceCtrl* ctrl, volatile int* abort_flag) {
   tcgen05_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned* count = &ctrl->barrier[0];
+    unsigned* gen = &ctrl->barrier[1];
+    const unsigned my_gen = ld_acquire_gpu(gen);
+    __threadfence();
+    const unsigned old = atomicAdd(count, 1u);
+    if (old == gridDim.x - 1) {
+      atomicExch(count, 0u);
+      __threadfence();
+      atomicAdd(gen, 1u);
+    } else {
+      const unsigned long long t0 = global_timer_ns();
+      while (ld_acquire_gpu(gen) == my_gen) {
+        __nanosleep(40);
+        if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+      }
+    }
+    __threadfence();
+  }
   __syncthreads();
   tcgen05_fence_after();
-  const uint32_t tmem_base = *tmem_holder;
+}
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t it = 0;
-      for (long long t = t_begin; t < t_end; ++t, ++it) {
-        const int s = it % NS;
-        if (!mbar_wait(&empty[s], ((it / NS) & 1) ^ 1, abort_flag)) break;
-        const int u = (int)(t / tpu), tt = (int)(t % tpu);
-        const int b = u / p.HG, hg = u % p.HG;
-        uint8_t* st = smem + s * STAGE;
-        mbar_arrive_expect_tx(&full[s], 4 * BOX);
-        int c0, c1;
-        box_coords<D>(0, hg, c0, c1);
-        tma_load_4d(st + 3 * BOX, &map_k, &full[s], c0, c1, tt * kTileState, b);
-        tma_load_4d(st + 0 * BOX, &map_v, &full[s], c0, c1, tt * kTileState, b);
-        box_coords<D>(1, hg, c0, c1);
-        tma_load_4d(st + 4 * BOX, &map_k, &full[s], c0, c1, tt * kTileState, b);
-        tma_load_4d(st + 1 * BOX, &map_v, &full[s], c0, c1, tt * kTileState, b);
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      uint32_t it = 0, seg = 0;
-      bool ok = true;
-      for (long long t = t_begin; t < t_end && ok; ++t, ++it) {
-        const int s = it % NS;
-        const int tt = (int)(t % tpu);
-        const bool seg_first = (t == t_begin) || tt == 0;
-        const bool seg_last = (t + 1 == t_end) || tt == tpu - 1;
-        const uint32_t acc = seg & 1;
-        if (seg_first) ok = mbar_wait(&tempty[acc], ((seg >> 1) & 1) ^ 1, abort_flag);
-        if (ok) ok = mbar_wait(&ready[s], (it / NS) & 1, abort_flag);
-        if (!ok) break;
-        tcgen05_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * kAccStride;
-        const uint32_t st = smem_u32(smem + s * STAGE);
-#pragma unroll
-        for (int kk = 0; kk < kTileState / 16; ++kk) {
-          const uint64_t a = make_smem_desc_sw128(st + 3 * BOX + kk * 2048, BOX, 1024);  // phi(K)^T, MN-major
-          const uint64_t bq = make_smem_desc_sw128(st + kk * 2048, BOX, 1024);           // [V | 1], MN-major
-          umma_bf16(d_tmem, a, bq, IDESC, (seg_first && kk == 0) ? 0u : 1u);
-        }
-        umma_commit(&empty[s]);
-        if (seg_last) { umma_commit(&tfull[acc]); ++seg; }
-      }
-    }
-  } else if (warp < 6) {
-    // ------------------------------------------------------------ ReLU pass over the K boxes
-    const int tr = threadIdx.x - kReluThread0;
-    uint32_t it = 0;
-    for (long long t = t_begin; t < t_end; ++t, ++it) {
-      const int s = it % NS;
-      if (!mbar_wait(&full[s], (it / NS) & 1, abort_flag)) break;
-      relu_pass<C::FEAT>(smem + s * STAGE + 3 * BOX, 2 * BOX / 16, BOX / 16, tr);
-      fence_proxy_async_smem();
-      mbar_arrive(&ready[s]);
-    }
-  } else {
-    // ------------------------------------------------------------ epilogue: accumulator -> partial record
-    const int wq = warp & 3;
-    const int i = wq * 32 + lane;           // accumulator lane = key feature within the group
-    const int g = i / D, il = i % D;        // head within the group, feature within the head
-    uint32_t seg = 0;
-    for (long long t = t_begin; t < t_end; ++t) {
-      const int tt = (int)(t % tpu);
-      const bool seg_last = (t + 1 == t_end) || tt == tpu - 1;
-      if (!seg_last) continue;
-      const uint32_t acc = seg & 1;
-      bool ok = mbar_wait(&tfull[acc], (seg >> 1) & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tcgen05_fence_after();
-      const int u = (int)(t / tpu);
-      const int b = u / p.HG, hg = u % p.HG;
-      const int h = hg * C::G + g;
-      const bool live = i < C::FEAT && h < p.H;
-      (void)b;
-      // record of this (CTA, unit) segment: G consecutive head-states in the library's layout
-      float* out = p.partials + ((size_t)(blockIdx.x + u) * C::G + g) * ((size_t)(D + 1) * D);
-      const uint32_t trow = tmem_base + acc * kAccStride + ((uint32_t)(wq * 32) << 16);
-#pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t r[32];
-        tmem_ld_x32(trow + cc * 32, r);
-        tmem_ld_wait();
-        if (live) {
-#pragma unroll
-          for (int x = 0; x < 32; ++x) {
-            const int j = cc * 32 + x;             // value feature within the group
-            const int jl = j - g * D;
-            if (jl >= 0 && jl < D) out[(size_t)jl * D + il] = __uint_as_float(r[x]);
-          }
-        }
-      }
-      uint32_t zr[4];
-      tmem_ld_x4(trow + 128, zr);
-      tmem_ld_wait();
-      if (live) out[(size_t)D * D + il] = __uint_as_float(zr[0]);
-      tcgen05_fence_before();
-      mbar_arrive(&tempty[acc]);
-      ++seg;
-    }
-  }
+// ---------------------------------------------------------------- reduce
+// This CTA's slice of the state: state[b][h][e] = (accumulate ? state : 0) + the partial records of
+// the head's unit, column CTAs first (ascending), then the trailing CTAs (ascending).
+__device__ __forceinline__ int trailing_cta_of(long long f, long long tot, int R) {
+  long long r = f * R / tot;
+  while (r + 1 < R && (r + 1) * tot / R <= f) ++r;
+  while (r > 0 && r * tot / R > f) --r;
+  return (int)r;
+}
 
-  // ------------------------------------------------------------ teardown
-  tcgen05_fence_before();
-  __syncthreads();
-  if (*abort_flag) {
-    if (threadIdx.x == 0) {
-      *p.status = LINATTN_ERR_TIMEOUT;
-      // loads still in flight target this CTA's shared memory: give each stage a bounded wait
-      for (int s = 0; s < NS; ++s)
-        for (int par = 0; par < 2; ++par)
-          for (int spin = 0; spin < 4096 && !mbar_try_wait(&full[s], par); ++spin) __nanosleep(64);
+template <int D>
+__device__ void reduce_slice(const FusedParams& p) {
+  using C = Cfg<D>;
+  constexpr int E = (D + 1) * D;
+  const Sched& s = p.sa;
+  const long long tot = (long long)p.B * p.H * E;
+  const long long i0 = (long long)blockIdx.x * tot / gridDim.x;
+  const long long i1 = (long long)(blockIdx.x + 1) * tot / gridDim.x;
+  const int ncol = s.P == 0 ? 0 : (s.P < (s.tpu + s.Lc - 1) / s.Lc ? s.P : (s.tpu + s.Lc - 1) / s.Lc);
+  const long long ttot = (long long)s.U * s.m;
+  for (long long idx = i0 + threadIdx.x; idx < i1; idx += kThreads) {
+    const int bh = (int)(idx / E), e = (int)(idx % E);
+    const int b = bh / p.H, h = bh % p.H;
+    const int u = b * p.HG + h / C::G, g = h % C::G;
+    const float* src = p.partials + (size_t)g * E + e;
+    float sum = p.accumulate ? __ldcg(p.state + idx) : 0.f;
+#pragma unroll 4
+    for (int c = 0; c < ncol; ++c) sum += __ldcg(src + (size_t)(c * s.U + u) * (C::G * E));
+    if (s.m > 0) {
+      const int r_lo = trailing_cta_of((long long)u * s.m, ttot, s.R);
+      const int r_hi = trailing_cta_of((long long)(u + 1) * s.m - 1, ttot, s.R);
+      for (int r = r_lo; r <= r_hi; ++r) sum += __ldcg(src + (size_t)(s.P * s.U + r + u) * (C::G * E));
     }
-    __syncthreads();
-  }
-  if (warp == 1) {
-    __syncwarp();
-    tcgen05_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    p.state[idx] = sum;
   }
 }
 
-// ============================================================================ reduce kernel
-// grid (ceil(E/256), B*H).  state[b][h][e] = (accumulate ? state : 0) + sum over the CTAs that
-// covered this head's group, in ascending CTA order.
-__device__ __forceinline__ long long cta_start(long long j, long long total, int grid) { return j * total / grid; }
-__device__ __forceinline__ int cta_of_tile(long long t, long long total, int grid) {
-  long long j = t * grid / total;
-  while (j + 1 < grid && cta_start(j + 1, total, grid) <= t) ++j;
-  while (j > 0 && cta_start(j, total, grid) > t) --j;
-  return (int)j;
-}
-
-__global__ void __launch_bounds__(256)
-umma_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state, int H, int HG, int G, int d,
-                   int tiles_per_unit, long long total_tiles, int grid_state, int accumulate) {
-  const long long E = (long long)(d + 1) * d;
-  const long long e = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (e >= E) return;
-  const int bh = blockIdx.y;
-  const int b = bh / H, h = bh % H;
-  const int u = b * HG + h / G, g = h % G;
-  const int j_lo = cta_of_tile((long long)u * tiles_per_unit, total_tiles, grid_state);
-  const int j_hi = cta_of_tile((long long)(u + 1) * tiles_per_unit - 1, total_tiles, grid_state);
-  float sum = accumulate ? state[(long long)bh * E + e] : 0.f;
-  for (int j = j_lo; j <= j_hi; ++j) sum += partials[((size_t)(j + u) * G + g) * E + e];
-  state[(long long)bh * E + e] = sum;
-}
-
-// ============================================================================ apply kernel
+// ---------------------------------------------------------------- S operand of the apply pass
 // Builds the B operand of the apply MMA for head group (b, hg) from the fp32 state: for every head
 // of the group, rows = value features (plus one row for z), K = key features, split into bf16 hi + lo.
 template <int D>
@@ -344,72 +295,124 @@ __device__ __forceinline__ void build_s_operand(uint8_t* s_op, const float* __re
   }
 }
 
+// ============================================================================ the kernel
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-umma_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o, UmmaParams p) {
+umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                  const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o, FusedParams p) {
   using C = Cfg<D>;
-  constexpr int NS = C::APPLY_SLOTS;
-  constexpr int SLOT = C::APPLY_SLOT_BYTES;
+  constexpr int NSA = C::STATE_STAGES;
+  constexpr int STAGE = C::STAGE_BYTES;
+  constexpr int NSC = C::APPLY_SLOTS;
+  constexpr int SLOT = C::SLOT_BYTES;
   constexpr int HALF = SLOT / 2;  // one 64-feature box of 128 tokens
-  constexpr uint32_t IDESC = make_idesc_bf16(128, C::NAPPLY, false, false);
+  constexpr uint32_t IDESC_A = make_idesc_bf16(128, C::NSTATE, true, true);
+  constexpr uint32_t IDESC_C = make_idesc_bf16(128, C::NAPPLY, false, false);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align1024(smem_raw);
-  uint8_t* s_op = smem;
-  uint8_t* slots = smem + C::S_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(slots + NS * SLOT);
-  uint64_t* full = bars;             // Q tile landed
-  uint64_t* ready = bars + NS;       // ReLU pass done
-  uint64_t* empty = bars + 2 * NS;   // O tile stored: slot reusable
-  uint64_t* tfull = bars + 3 * NS;   // [2] accumulator complete
-  uint64_t* tempty = tfull + 2;      // [2] accumulator drained
-  uint64_t* s_ready = tempty + 2;    // S operand of the current segment is in shared memory
-  uint64_t* seg_done = s_ready + 1;  // every MMA of the finished segment is complete
-  uint64_t* o_staged = seg_done + 1; // the 128 epilogue threads have written their O rows
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(o_staged + 1);
+  uint8_t* s_op = smem;                    // apply pass: S operand ...
+  uint8_t* slots = smem + C::S_BYTES;      // ... and the Q/O slots; the state pass stages cover both
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::DATA_BYTES);
+  // state pass
+  uint64_t* a_full = bars;                 // TMA landed
+  uint64_t* a_ready = a_full + NSA;        // ReLU pass done
+  uint64_t* a_empty = a_ready + NSA;       // MMAs that read the stage are complete
+  uint64_t* a_tfull = a_empty + NSA;       // [2] accumulator complete
+  uint64_t* a_tempty = a_tfull + 2;        // [2] accumulator drained by the epilogue
+  uint64_t* a_done = a_tempty + 2;         // every MMA of the state pass is complete: stages are free
+  // apply pass
+  uint64_t* c_full = a_done + 1;           // Q tile landed
+  uint64_t* c_ready = c_full + NSC;        // ReLU pass done
+  uint64_t* c_empty = c_ready + NSC;       // O tile read out by its TMA store: slot reusable
+  uint64_t* c_staged = c_empty + NSC;      // the 128 epilogue threads have written their O rows
+  uint64_t* c_tfull = c_staged + NSC;      // [2] accumulator complete
+  uint64_t* c_tempty = c_tfull + 2;        // [2] accumulator drained
+  uint64_t* s_ready = c_tempty + 2;        // S operand of the current segment is in shared memory
+  uint64_t* seg_done = s_ready + 1;        // every MMA of the finished segment is complete
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(seg_done + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  static_assert((3 * NSA + 5 + 4 * NSC + 6) * 8 + 8 <= C::BAR_BYTES, "barrier block too small");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long t_begin = (long long)blockIdx.x * p.total_tiles / gridDim.x;
-  const long long t_end = (long long)(blockIdx.x + 1) * p.total_tiles / gridDim.x;
-  const int tpu = p.tiles_per_unit;
+  const Work wa = p.do_state ? work_of(p.sa, blockIdx.x) : work_of(p.sa, 0x7fffffff);
+  const Work wc = p.do_apply ? work_of(p.sc, blockIdx.x) : work_of(p.sc, 0x7fffffff);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&ready[s], 128); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 128); }
+    for (int s = 0; s < NSA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_ready[s], 128); mbar_init(&a_empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&a_tfull[b], 1); mbar_init(&a_tempty[b], 128); }
+    mbar_init(a_done, 1);
+    for (int s = 0; s < NSC; ++s) {
+      mbar_init(&c_full[s], 1); mbar_init(&c_ready[s], 128); mbar_init(&c_empty[s], 1); mbar_init(&c_staged[s], 128);
+    }
+    for (int b = 0; b < 2; ++b) { mbar_init(&c_tfull[b], 1); mbar_init(&c_tempty[b], 128); }
     mbar_init(s_ready, 256);
     mbar_init(seg_done, 128);
-    mbar_init(o_staged, 128);
     *abort_flag = 0;
     fence_mbar_init();
+    prefetch_tensormap(&map_k);
+    prefetch_tensormap(&map_v);
     prefetch_tensormap(&map_q);
     prefetch_tensormap(&map_o);
   }
-  // rows of the S operand that no head ever writes (padding rows, cross-head blocks) stay zero
-  for (int idx = threadIdx.x; idx < C::S_BYTES / 16; idx += kThreads)
-    *reinterpret_cast<uint4*>(s_op + idx * 16) = make_uint4(0, 0, 0, 0);
-  fence_proxy_async_smem();
+  if (C::ONES_BOX && wa.f1 > wa.f0) {
+    // the constant "ones" chunk of every stage: value columns 128..191 of B, of which column 128 is 1
+    for (int idx = threadIdx.x; idx < NSA * (kBox / 16); idx += kThreads) {
+      const int s = idx / (kBox / 16), c = idx % (kBox / 16);
+      const int row = c >> 3, phys = c & 7;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if ((phys ^ (row & 7)) == 0) val.x = 0x3F80u;  // bf16 1.0 in element 0 of logical chunk 0
+      *reinterpret_cast<uint4*>(smem + s * STAGE + 2 * kBox + c * 16) = val;
+    }
+    fence_proxy_async_smem();
+  }
   if (warp == 1) { tmem_alloc(tmem_holder, kTmemCols); tmem_relinquish(); }
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
+  // apply-pass producer state lives across the grid barriers (the first tiles are fetched before them)
+  TileWalk cw(wc);
+  uint32_t c_it = 0;
+  auto load_q_tile = [&]() -> bool {
+    const int s = c_it % NSC;
+    if (!mbar_wait(&c_empty[s], ((c_it / NSC) & 1) ^ 1, abort_flag)) return false;
+    const int u = cw.unit(), b = u / p.HG, hg = u % p.HG;
+    uint8_t* sl = slots + s * SLOT;
+    mbar_arrive_expect_tx(&c_full[s], SLOT);
+    int c0, c1;
+    box_coords<D>(0, hg, c0, c1);
+    tma_load_4d(sl, &map_q, &c_full[s], c0, c1, cw.tile() * kTileApply, b);
+    box_coords<D>(1, hg, c0, c1);
+    tma_load_4d(sl + HALF, &map_q, &c_full[s], c0, c1, cw.tile() * kTileApply, b);
+    cw.next();
+    ++c_it;
+    return true;
+  };
+
+  // ==================================================================== state pass
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer: Q tiles
+    // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t it = 0;
-      for (long long t = t_begin; t < t_end; ++t, ++it) {
-        const int s = it % NS;
-        if (!mbar_wait(&empty[s], ((it / NS) & 1) ^ 1, abort_flag)) break;
-        const int u = (int)(t / tpu), tt = (int)(t % tpu);
-        const int b = u / p.HG, hg = u % p.HG;
-        uint8_t* sl = slots + s * SLOT;
-        mbar_arrive_expect_tx(&full[s], SLOT);
+      for (TileWalk t(wa); !t.done(); t.next(), ++it) {
+        const int s = it % NSA;
+        if (!mbar_wait(&a_empty[s], ((it / NSA) & 1) ^ 1, abort_flag)) break;
+        const int u = t.unit(), b = u / p.HG, hg = u % p.HG;
+        uint8_t* st = smem + s * STAGE;
+        mbar_arrive_expect_tx(&a_full[s], 4 * kBox);
         int c0, c1;
         box_coords<D>(0, hg, c0, c1);
-        tma_load_4d(sl, &map_q, &full[s], c0, c1, tt * kTileApply, b);
+        tma_load_4d(st + C::KOFF, &map_k, &a_full[s], c0, c1, t.tile() * kTileState, b);
+        tma_load_4d(st, &map_v, &a_full[s], c0, c1, t.tile() * kTileState, b);
         box_coords<D>(1, hg, c0, c1);
-        tma_load_4d(sl + HALF, &map_q, &full[s], c0, c1, tt * kTileApply, b);
+        tma_load_4d(st + C::KOFF + kBox, &map_k, &a_full[s], c0, c1, t.tile() * kTileState, b);
+        tma_load_4d(st + kBox, &map_v, &a_full[s], c0, c1, t.tile() * kTileState, b);
+      }
+      // the stages are free once every MMA of this pass is complete: start on the Q tiles now
+      if (wc.f1 > wc.f0 && mbar_wait(a_done, 0, abort_flag)) {
+        while (!cw.done() && c_it < (uint32_t)NSC)
+          if (!load_q_tile()) break;
       }
     }
   } else if (warp == 1) {
@@ -417,13 +420,120 @@ umma_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (lane == 0) {
       uint32_t it = 0, seg = 0;
       bool ok = true;
-      for (long long t = t_begin; t < t_end && ok; ++t, ++it) {
-        const int s = it % NS;
-        const int tt = (int)(t % tpu);
-        if (t == t_begin || tt == 0) { ok = mbar_wait(s_ready, seg & 1, abort_flag); ++seg; }
+      for (TileWalk t(wa); !t.done() && ok; t.next(), ++it) {
+        const int s = it % NSA;
+        const bool seg_first = t.seg_first();
+        const uint32_t acc = seg & 1;
+        if (seg_first) ok = mbar_wait(&a_tempty[acc], ((seg >> 1) & 1) ^ 1, abort_flag);
+        if (ok) ok = mbar_wait(&a_ready[s], (it / NSA) & 1, abort_flag);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * kAccStride;
+        const uint32_t st = smem_u32(smem + s * STAGE);
+#pragma unroll
+        for (int kk = 0; kk < kTileState / 16; ++kk) {
+          const uint64_t a = make_smem_desc_sw128(st + C::KOFF + kk * 2048, kBox, 1024);  // phi(K)^T, MN-major
+          const uint64_t bq = make_smem_desc_sw128(st + kk * 2048, kBox, 1024);           // [V | 1], MN-major
+          umma_bf16(d_tmem, a, bq, IDESC_A, (seg_first && kk == 0) ? 0u : 1u);
+        }
+        umma_commit(&a_empty[s]);
+        if (t.seg_last()) { umma_commit(&a_tfull[acc]); ++seg; }
+      }
+      if (it > 0) umma_commit(a_done); else mbar_arrive(a_done);
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------ ReLU pass over the K boxes
+    const int tr = threadIdx.x - kReluThread0;
+    uint32_t it = 0;
+    for (TileWalk t(wa); !t.done(); t.next(), ++it) {
+      const int s = it % NSA;
+      if (!mbar_wait(&a_full[s], (it / NSA) & 1, abort_flag)) break;
+      uint8_t* st = smem + s * STAGE;
+      relu_pass<C::FEAT>(st + C::KOFF, 2 * kBox / 16, kBox / 16, tr);
+      if (!C::ONES_BOX && tr < kTileState) {
+        // value column 112 := 1 (logical chunk 6 of the second V box, element 0), so z is accumulator column 112
+        *reinterpret_cast<uint16_t*>(st + kBox + tr * kRowBytes + ((6 ^ (tr & 7)) << 4)) = 0x3F80u;
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(&a_ready[s]);
+    }
+  } else if (warp < kStoreWarp) {
+    // ------------------------------------------------------------ epilogue: accumulator -> partial record
+    const int wq = warp & 3;
+    const int i = wq * 32 + lane;           // accumulator lane = key feature within the group
+    const int g = i / D, il = i % D;        // head within the group, feature within the head
+    uint32_t seg = 0;
+    for (TileWalk t(wa); !t.done(); t.next()) {
+      if (!t.seg_last()) continue;
+      const uint32_t acc = seg & 1;
+      bool ok = mbar_wait(&a_tfull[acc], (seg >> 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tcgen05_fence_after();
+      const int u = t.unit(), hg = u % p.HG;
+      const int h = hg * C::G + g;
+      const bool live = i < C::FEAT && h < p.H;
+      // record of this (CTA, unit) segment: G consecutive head-states in the library's layout
+      float* out = p.partials + ((size_t)t.record() * C::G + g) * ((size_t)(D + 1) * D);
+      const uint32_t trow = tmem_base + acc * kAccStride + ((uint32_t)(wq * 32) << 16);
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t r[32];
+        tmem_ld_x32(trow + cc * 32, r);
+        tmem_ld_wait();
+        if (live) {
+#pragma unroll
+          for (int x = 0; x < 32; ++x) {
+            const int j = cc * 32 + x;             // value feature within the group
+            const int jl = j - g * D;
+            if (jl >= 0 && jl < D) out[(size_t)jl * D + il] = __uint_as_float(r[x]);
+            if (!C::ONES_BOX && j == C::ZCOL) out[(size_t)D * D + il] = __uint_as_float(r[x]);
+          }
+        }
+      }
+      if (C::ONES_BOX) {
+        uint32_t zr[4];
+        tmem_ld_x4(trow + C::ZCOL, zr);
+        tmem_ld_wait();
+        if (live) out[(size_t)D * D + il] = __uint_as_float(zr[0]);
+      }
+      tcgen05_fence_before();
+      mbar_arrive(&a_tempty[acc]);
+      ++seg;
+    }
+  }
+
+  // ==================================================================== reduce
+  if (p.do_state) {
+    grid_barrier(p.ctrl, abort_flag);
+    if (!*abort_flag) reduce_slice<D>(p);
+    if (p.do_apply) grid_barrier(p.ctrl, abort_flag);
+  }
+  if (C::G > 1 && wc.f1 > wc.f0) {
+    // cross-head blocks of the packed S operand are never written by a head: they must read as zero
+    for (int idx = threadIdx.x; idx < C::S_BYTES / 16; idx += kThreads)
+      *reinterpret_cast<uint4*>(s_op + idx * 16) = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+  }
+
+  // ==================================================================== apply pass
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer: the remaining Q tiles
+    if (lane == 0) {
+      while (!cw.done())
+        if (!load_q_tile()) break;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, seg = 0;
+      bool ok = true;
+      for (TileWalk t(wc); !t.done() && ok; t.next(), ++it) {
+        const int s = it % NSC;
+        if (t.seg_first()) { ok = mbar_wait(s_ready, seg & 1, abort_flag); ++seg; }
         const uint32_t acc = it & 1;
-        if (ok) ok = mbar_wait(&tempty[acc], ((it >> 1) & 1) ^ 1, abort_flag);
-        if (ok) ok = mbar_wait(&ready[s], (it / NS) & 1, abort_flag);
+        if (ok) ok = mbar_wait(&c_tempty[acc], ((it >> 1) & 1) ^ 1, abort_flag);
+        if (ok) ok = mbar_wait(&c_ready[s], (it / NSC) & 1, abort_flag);
         if (!ok) break;
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kAccStride;
@@ -436,10 +546,10 @@ umma_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           const uint64_t a = make_smem_desc_sw128(a0 + koff, 16, 1024);                           // phi(Q), K-major
           const uint64_t bh = make_smem_desc_sw128(b0 + boff, 16, 1024);                          // S hi
           const uint64_t bl = make_smem_desc_sw128(b0 + 2 * C::SBOX_BYTES + boff, 16, 1024);      // S lo
-          umma_bf16(d_tmem, a, bh, IDESC, k == 0 ? 0u : 1u);
-          umma_bf16(d_tmem, a, bl, IDESC, 1u);
+          umma_bf16(d_tmem, a, bh, IDESC_C, k == 0 ? 0u : 1u);
+          umma_bf16(d_tmem, a, bl, IDESC_C, 1u);
         }
-        umma_commit(&tfull[acc]);
+        umma_commit(&c_tfull[acc]);
       }
     }
   } else if (warp < 6) {
@@ -447,46 +557,44 @@ umma_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int tr = threadIdx.x - kReluThread0;
     uint32_t it = 0, seg = 0;
     bool ok = true;
-    for (long long t = t_begin; t < t_end && ok; ++t, ++it) {
-      const int s = it % NS;
-      const int tt = (int)(t % tpu);
-      if (t == t_begin || tt == 0) {
+    for (TileWalk t(wc); !t.done() && ok; t.next(), ++it) {
+      const int s = it % NSC;
+      if (t.seg_first()) {
         // the previous segment's MMAs must be done before its S operand is overwritten
         if (seg > 0) ok = mbar_wait(seg_done, (seg - 1) & 1, abort_flag);
         if (!ok) break;
-        const int u = (int)(t / tpu);
-        build_s_operand<D>(s_op, p.state_in, u / p.HG, u % p.HG, p.H, tr, 256);
+        const int u = t.unit();
+        build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, tr, 256);
         fence_proxy_async_smem();
         mbar_arrive(s_ready);
         ++seg;
       }
-      if (!mbar_wait(&full[s], (it / NS) & 1, abort_flag)) break;
+      if (!mbar_wait(&c_full[s], (it / NSC) & 1, abort_flag)) break;
       relu_pass<C::FEAT>(slots + s * SLOT, SLOT / 16, HALF / 16, tr);
       fence_proxy_async_smem();
-      mbar_arrive(&ready[s]);
+      mbar_arrive(&c_ready[s]);
     }
-  } else {
-    // ------------------------------------------------------------ epilogue: divide, round, store
-    const int te = threadIdx.x - kEpiThread0;
+  } else if (warp < kStoreWarp) {
+    // ------------------------------------------------------------ epilogue: divide, round, stage the O tile
     const int wq = warp & 3;
+    const int te = threadIdx.x - kEpiThread0;
     const int r = wq * 32 + lane;  // accumulator lane = token row of the tile
     uint32_t it = 0;
-    for (long long t = t_begin; t < t_end; ++t, ++it) {
-      const int s = it % NS;
-      const int u = (int)(t / tpu), tt = (int)(t % tpu);
-      const int b = u / p.HG, hg = u % p.HG;
-      if (t == t_begin || tt == 0) {
+    for (TileWalk t(wc); !t.done(); t.next(), ++it) {
+      const int s = it % NSC;
+      if (t.seg_first()) {
         // this thread has seen the last accumulator of the previous segment complete: S may be rebuilt
-        build_s_operand<D>(s_op, p.state_in, b, hg, p.H, 128 + te, 256);
+        const int u = t.unit();
+        build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, 128 + te, 256);
         fence_proxy_async_smem();
         mbar_arrive(s_ready);
       }
       const uint32_t acc = it & 1;
-      bool ok = mbar_wait(&tfull[acc], (it >> 1) & 1, abort_flag);
+      bool ok = mbar_wait(&c_tfull[acc], (it >> 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      if ((t + 1 == t_end) || tt == tpu - 1) mbar_arrive(seg_done);
+      if (t.seg_last()) mbar_arrive(seg_done);
       const uint32_t trow = tmem_base + acc * kAccStride + ((uint32_t)(wq * 32) << 16);
       uint32_t dn[4];
       tmem_ld_x4(trow + C::ZROW, dn);
@@ -503,7 +611,7 @@ umma_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         tmem_ld_wait();
         if (cc == 3 || (cc + 1) * 32 >= C::FEAT) {  // last read of this accumulator: hand it back to the MMA warp
           tcgen05_fence_before();
-          mbar_arrive(&tempty[acc]);
+          mbar_arrive(&c_tempty[acc]);
         }
         const float ri = rinv[(cc * 32) / D < C::G ? (cc * 32) / D : 0];
 #pragma unroll
@@ -519,24 +627,28 @@ umma_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
       }
       fence_proxy_async_smem();
-      mbar_arrive(o_staged);
-      bool stored = true;
-      if (te == 0) {
-        stored = mbar_wait(o_staged, it & 1, abort_flag);
-        if (stored) {
-          int c0, c1;
-          box_coords<D>(0, hg, c0, c1);
-          tma_store_4d(&map_o, sl, c0, c1, tt * kTileApply, b);
-          box_coords<D>(1, hg, c0, c1);
-          tma_store_4d(&map_o, sl + HALF, c0, c1, tt * kTileApply, b);
-          tma_store_commit();
-          tma_store_wait_read();
-          mbar_arrive(&empty[s]);
-        }
-      }
-      if (!__all_sync(0xffffffffu, stored)) break;  // leave the loop as a whole warp
+      mbar_arrive(&c_staged[s]);
     }
-    if (te == 0) tma_store_wait_all();
+  } else {
+    // ------------------------------------------------------------ store warp: O tiles out, slots back to the producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (TileWalk t(wc); !t.done(); t.next(), ++it) {
+        const int s = it % NSC;
+        if (!mbar_wait(&c_staged[s], (it / NSC) & 1, abort_flag)) break;
+        const int u = t.unit(), b = u / p.HG, hg = u % p.HG;
+        uint8_t* sl = slots + s * SLOT;
+        int c0, c1;
+        box_coords<D>(0, hg, c0, c1);
+        tma_store_4d(&map_o, sl, c0, c1, t.tile() * kTileApply, b);
+        box_coords<D>(1, hg, c0, c1);
+        tma_store_4d(&map_o, sl + HALF, c0, c1, t.tile() * kTileApply, b);
+        tma_store_commit();
+        tma_store_wait_read();
+        mbar_arrive(&c_empty[s]);
+      }
+      tma_store_wait_all();
+    }
   }
 
   // ------------------------------------------------------------ teardown
@@ -544,10 +656,12 @@ umma_apply_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   __syncthreads();
   if (*abort_flag) {
     if (threadIdx.x == 0) {
-      *p.status = LINATTN_ERR_TIMEOUT;
-      for (int s = 0; s < NS; ++s)
+      p.ctrl->status = LINATTN_ERR_TIMEOUT;
+      // loads still in flight target this CTA's shared memory: give each stage a bounded wait
+      for (int s = 0; s < NSA + NSC; ++s)
         for (int par = 0; par < 2; ++par)
-          for (int spin = 0; spin < 4096 && !mbar_try_wait(&full[s], par); ++spin) __nanosleep(64);
+          for (int spin = 0; spin < 4096 && !mbar_try_wait(s < NSA ? &a_full[s] : &c_full[s - NSA], par); ++spin)
+            __nanosleep(64);
     }
     __syncthreads();
   }
@@ -589,78 +703,67 @@ bool make_map(CUtensorMap* map, const Problem& p, const void* base, int box_d, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// SM count of the current device (0: not an sm_100 device, or no cooperative launch).
 int sm_count() {
   static int cached[64] = {0};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
   if (!cached[dev]) {
-    int n = 0, major = 0;
+    int n = 0, major = 0, coop = 0;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || major != 10) return 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return 0;
     cached[dev] = n > kMaxCtas ? kMaxCtas : n;
   }
   return cached[dev];
 }
 
-inline int groups_of(int d) { return d == 32 ? 4 : d == 64 ? 2 : 1; }
+inline int groups_of(int d) { return d == 64 ? 2 : 1; }
 
 template <int D>
-int launch_state(const Problem& p, const void* k, const void* v, float* state, bool accumulate, float* partials,
-                 int* status, cudaStream_t stream) {
+int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
   using C = Cfg<D>;
   const int sms = sm_count();
   if (!sms) return LINATTN_ERR_CUDA;
-  UmmaParams up{};
-  up.B = p.B; up.H = p.H; up.HG = (p.H + C::G - 1) / C::G; up.N = p.N;
-  up.tiles_per_unit = (int)((p.N + kTileState - 1) / kTileState);
-  up.total_tiles = (long long)p.B * up.HG * up.tiles_per_unit;
-  up.partials = partials; up.status = status;
-  const int grid = (int)(up.total_tiles < sms ? up.total_tiles : sms);
-  CUtensorMap mk, mv;
-  if (!make_map(&mk, p, k, C::BOX_D, C::BOX_H, kTileState) || !make_map(&mv, p, v, C::BOX_D, C::BOX_H, kTileState))
-    return LINATTN_ERR_CUDA;
+  const bool do_state = c.k != nullptr, do_apply = c.q != nullptr;
+  FusedParams fp{};
+  fp.B = p.B; fp.H = p.H; fp.HG = (p.H + C::G - 1) / C::G;
+  const int U = p.B * fp.HG;
+  fp.sa = make_sched(U, (p.N + kTileState - 1) / kTileState, sms);
+  fp.sc = make_sched(U, (p.N + kTileApply - 1) / kTileApply, sms);
+  fp.do_state = do_state; fp.do_apply = do_apply; fp.accumulate = c.accumulate ? 1 : 0;
+  fp.state = c.state;
+  fp.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + LINATTN_WORKSPACE_CTRL_BYTES);
+  fp.eps = c.eps;
+  fp.ctrl = static_cast<WorkspaceCtrl*>(workspace);
+  int grid = 0;
+  if (do_state) grid = fp.sa.grid;
+  if (do_apply && fp.sc.grid > grid) grid = fp.sc.grid;
+  CUtensorMap mk, mv, mq, mo;
+  if (do_state) {
+    if (!make_map(&mk, p, c.k, C::BOX_D, C::BOX_H, kTileState) || !make_map(&mv, p, c.v, C::BOX_D, C::BOX_H, kTileState))
+      return LINATTN_ERR_CUDA;
+  }
+  if (do_apply) {
+    if (!make_map(&mq, p, c.q, C::BOX_D, C::BOX_H, kTileApply) || !make_map(&mo, p, c.o, C::BOX_D, C::BOX_H, kTileApply))
+      return LINATTN_ERR_CUDA;
+  } else {
+    mq = mk; mo = mk;  // never dereferenced
+  }
+  if (!do_state) { mk = mq; mv = mq; }
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(umma_state_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::STATE_SMEM) !=
+    if (cudaFuncSetAttribute(umma_fused_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM) !=
         cudaSuccess)
       return LINATTN_ERR_CUDA;
     attr_set = true;
   }
-  umma_state_kernel<D><<<grid, kThreads, C::STATE_SMEM, stream>>>(mk, mv, up);
-  if (cudaGetLastError() != cudaSuccess) return LINATTN_ERR_CUDA;
-  const long long E = p.state_elems();
-  dim3 rgrid((unsigned)((E + 255) / 256), (unsigned)(p.B * p.H));
-  umma_reduce_kernel<<<rgrid, 256, 0, stream>>>(partials, state, p.H, up.HG, C::G, D, up.tiles_per_unit, up.total_tiles,
-                                                grid, accumulate ? 1 : 0);
-  count_launches(2);
-  return cudaGetLastError() == cudaSuccess ? LINATTN_OK : LINATTN_ERR_CUDA;
-}
-
-template <int D>
-int launch_apply(const Problem& p, const void* q, const float* state, void* o, float eps, int* status,
-                 cudaStream_t stream) {
-  using C = Cfg<D>;
-  const int sms = sm_count();
-  if (!sms) return LINATTN_ERR_CUDA;
-  UmmaParams up{};
-  up.B = p.B; up.H = p.H; up.HG = (p.H + C::G - 1) / C::G; up.N = p.N;
-  up.tiles_per_unit = (int)((p.N + kTileApply - 1) / kTileApply);
-  up.total_tiles = (long long)p.B * up.HG * up.tiles_per_unit;
-  up.state_in = state; up.eps = eps; up.status = status;
-  const int grid = (int)(up.total_tiles < sms ? up.total_tiles : sms);
-  CUtensorMap mq, mo;
-  if (!make_map(&mq, p, q, C::BOX_D, C::BOX_H, kTileApply) || !make_map(&mo, p, o, C::BOX_D, C::BOX_H, kTileApply))
-    return LINATTN_ERR_CUDA;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(umma_apply_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::APPLY_SMEM) !=
-        cudaSuccess)
-      return LINATTN_ERR_CUDA;
-    attr_set = true;
-  }
-  umma_apply_kernel<D><<<grid, kThreads, C::APPLY_SMEM, stream>>>(mq, mo, up);
+  void* args[] = {&mk, &mv, &mq, &mo, &fp};
+  const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D>, dim3(grid), dim3(kThreads), args,
+                                                    C::SMEM, stream);
+  if (e != cudaSuccess) { cudaGetLastError(); return LINATTN_ERR_CUDA; }
   count_launches(1);
-  return cudaGetLastError() == cudaSuccess ? LINATTN_OK : LINATTN_ERR_CUDA;
+  return LINATTN_OK;
 }
 
 }  // namespace
@@ -672,37 +775,19 @@ bool umma_supported(const Problem& p) {
          p.N < (1ll << 31) && p.sh * 2 < (1ll << 40) && p.sn * 2 < (1ll << 40) && p.sb * 2 < (1ll << 40);
 }
 
-// One partial record (G head-states) per (CTA, unit) segment: at most kMaxCtas + units records.
+// One partial record (G head-states) per (CTA, unit) segment of the state pass: at most kMaxCtas + units.
 size_t umma_partial_bytes(const Problem& p) {
   const int G = groups_of(p.d);
   const size_t units = (size_t)p.B * ((p.H + G - 1) / G);
   return ((size_t)kMaxCtas + units) * G * (size_t)p.state_elems() * sizeof(float);
 }
 
-int umma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate, void* workspace,
-               cudaStream_t stream) {
-  if (p.N == 0) {
-    if (accumulate) return LINATTN_OK;
-    return cudaMemsetAsync(state_out, 0, sizeof(float) * p.state_elems() * p.units(), stream) == cudaSuccess
-               ? LINATTN_OK : LINATTN_ERR_CUDA;
-  }
-  float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + LINATTN_WORKSPACE_CTRL_BYTES);
-  int* status = &static_cast<WorkspaceCtrl*>(workspace)->status;
+int umma_run(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
+  if (p.N == 0 || (!c.k && !c.q)) return LINATTN_OK;
   switch (p.d) {
-    case 64: return launch_state<64>(p, k, v, state_out, accumulate, partials, status, stream);
-    case 112: return launch_state<112>(p, k, v, state_out, accumulate, partials, status, stream);
-    case 128: return launch_state<128>(p, k, v, state_out, accumulate, partials, status, stream);
-  }
-  return LINATTN_ERR_UNSUPPORTED;
-}
-
-int umma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, int* status,
-               cudaStream_t stream) {
-  if (p.N == 0) return LINATTN_OK;
-  switch (p.d) {
-    case 64: return launch_apply<64>(p, q, state, o, eps, status, stream);
-    case 112: return launch_apply<112>(p, q, state, o, eps, status, stream);
-    case 128: return launch_apply<128>(p, q, state, o, eps, status, stream);
+    case 64: return launch_fused<64>(p, c, workspace, stream);
+    case 112: return launch_fused<112>(p, c, workspace, stream);
+    case 128: return launch_fused<128>(p, c, workspace, stream);
   }
   return LINATTN_ERR_UNSUPPORTED;
 }
