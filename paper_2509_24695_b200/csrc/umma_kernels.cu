@@ -168,21 +168,33 @@ __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
   return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~(uintptr_t)1023);
 }
 
-// In-place ReLU over `nchunks` 16-byte chunks starting at `base`, 128 threads, thread `t`.
-// With FEAT = 112 the chunks that hold only the zero padding (features 112..127) are skipped.
-template <int FEAT>
-__device__ __forceinline__ void relu_pass(uint8_t* base, int nchunks, int chunks_per_box, int t) {
-  for (int idx = t; idx < nchunks; idx += 128) {
-    if (FEAT < 128) {
-      const int in_box = idx % chunks_per_box;
-      const int box = (idx / chunks_per_box) & 1;
-      const int row = in_box >> 3, phys = in_box & 7;
-      if (box == 1 && (((phys ^ (row & 7)) << 3) + 64) >= FEAT) continue;
+// In-place ReLU over the two 64-feature boxes (ROWS token rows of 128 bytes each, 128-byte swizzle) of a
+// tile, 128 threads, thread `t`.  A thread owns one 16-byte column position of rows t/8 + 16*i; with the
+// 128-byte swizzle the logical chunk at that position is the same for all of its rows, so with FEAT = 112
+// a thread whose chunk of the second box holds only zero padding (features 112..127) skips that box.
+// All loads of a box are issued before the first store.
+template <int FEAT, int ROWS>
+__device__ __forceinline__ void relu_pass(uint8_t* box0, uint8_t* box1, int t) {
+  const int row0 = t >> 3, pc = t & 7;
+  const int lc = pc ^ (row0 & 7);
+  uint8_t* p0 = box0 + row0 * kRowBytes + pc * 16;
+  uint8_t* p1 = box1 + row0 * kRowBytes + pc * 16;
+  uint4 x[ROWS / 16];
+#pragma unroll
+  for (int i = 0; i < ROWS / 16; ++i) x[i] = *reinterpret_cast<uint4*>(p0 + i * 16 * kRowBytes);
+#pragma unroll
+  for (int i = 0; i < ROWS / 16; ++i) {
+    x[i].x = relu_bf16x2(x[i].x); x[i].y = relu_bf16x2(x[i].y); x[i].z = relu_bf16x2(x[i].z); x[i].w = relu_bf16x2(x[i].w);
+    *reinterpret_cast<uint4*>(p0 + i * 16 * kRowBytes) = x[i];
+  }
+  if (FEAT >= 128 || 64 + lc * 8 < FEAT) {
+#pragma unroll
+    for (int i = 0; i < ROWS / 16; ++i) x[i] = *reinterpret_cast<uint4*>(p1 + i * 16 * kRowBytes);
+#pragma unroll
+    for (int i = 0; i < ROWS / 16; ++i) {
+      x[i].x = relu_bf16x2(x[i].x); x[i].y = relu_bf16x2(x[i].y); x[i].z = relu_bf16x2(x[i].z); x[i].w = relu_bf16x2(x[i].w);
+      *reinterpret_cast<uint4*>(p1 + i * 16 * kRowBytes) = x[i];
     }
-    uint4* p = reinterpret_cast<uint4*>(base + (size_t)idx * 16);
-    uint4 x = *p;
-    x.x = relu_bf16x2(x.x); x.y = relu_bf16x2(x.y); x.z = relu_bf16x2(x.z); x.w = relu_bf16x2(x.w);
-    *p = x;
   }
 }
 
@@ -193,27 +205,23 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
   return v;
 }
 
-// All CTAs of the (cooperatively launched, hence co-resident) grid meet here.  Sense-reversing and
-// self-resetting: the last CTA to arrive zeroes the counter and bumps the generation word the others
-// poll.  The poll is bounded (about a second); on expiry the CTA raises its abort flag and goes on
-// to the teardown.
+// All CTAs of the (cooperatively launched, hence co-resident) grid meet here.  One word holds the
+// arrival count (low 16 bits) and a generation (high 16 bits): the last CTA to arrive clears the count
+// and bumps the generation with one more atomic, the others poll the word until the generation
+// moves.  The poll is bounded (about a second); on expiry the CTA raises its abort flag and goes on to
+// the teardown.
 __device__ __forceinline__ void grid_barrier(WorkspaceCtrl* ctrl, volatile int* abort_flag) {
   tcgen05_fence_before();
   __syncthreads();
   if (threadIdx.x == 0) {
-    unsigned* count = &ctrl->barrier[0];
-    unsigned* gen = &ctrl->barrier[1];
-    const unsigned my_gen = ld_acquire_gpu(gen);
+    unsigned* word = &ctrl->barrier[0];
     __threadfence();
-    const unsigned old = atomicAdd(count, 1u);
-    if (old == gridDim.x - 1) {
-      atomicExch(count, 0u);
-      __threadfence();
-      atomicAdd(gen, 1u);
+    const unsigned old = atomicAdd(word, 1u);
+    if ((old & 0xFFFFu) == gridDim.x - 1) {
+      atomicAdd(word, 0x10000u - gridDim.x);
     } else {
       const unsigned long long t0 = global_timer_ns();
-      while (ld_acquire_gpu(gen) == my_gen) {
-        __nanosleep(40);
+      while ((ld_acquire_gpu(word) >> 16) == (old >> 16)) {
         if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
       }
     }
@@ -233,30 +241,50 @@ __device__ __forceinline__ int trailing_cta_of(long long f, long long tot, int R
   return (int)r;
 }
 
+__device__ __forceinline__ void add4(float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+
 template <int D>
 __device__ void reduce_slice(const FusedParams& p) {
   using C = Cfg<D>;
-  constexpr int E = (D + 1) * D;
+  constexpr int E4 = (D + 1) * D / 4;  // float4 per head state
+  constexpr int REC4 = C::G * E4;      // float4 per partial record
   const Sched& s = p.sa;
-  const long long tot = (long long)p.B * p.H * E;
+  const long long tot = (long long)p.B * p.H * E4;
   const long long i0 = (long long)blockIdx.x * tot / gridDim.x;
   const long long i1 = (long long)(blockIdx.x + 1) * tot / gridDim.x;
   const int ncol = s.P == 0 ? 0 : (s.P < (s.tpu + s.Lc - 1) / s.Lc ? s.P : (s.tpu + s.Lc - 1) / s.Lc);
   const long long ttot = (long long)s.U * s.m;
+  float4* state4 = reinterpret_cast<float4*>(p.state);
   for (long long idx = i0 + threadIdx.x; idx < i1; idx += kThreads) {
-    const int bh = (int)(idx / E), e = (int)(idx % E);
+    const int bh = (int)(idx / E4), e = (int)(idx % E4);
     const int b = bh / p.H, h = bh % p.H;
     const int u = b * p.HG + h / C::G, g = h % C::G;
-    const float* src = p.partials + (size_t)g * E + e;
-    float sum = p.accumulate ? __ldcg(p.state + idx) : 0.f;
-#pragma unroll 4
-    for (int c = 0; c < ncol; ++c) sum += __ldcg(src + (size_t)(c * s.U + u) * (C::G * E));
+    const float4* src = reinterpret_cast<const float4*>(p.partials) + (size_t)g * E4 + e;
+    float4 sum = p.accumulate ? __ldcg(state4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+    // the loads of a batch are independent and issued together; the adds keep the fixed order
+    for (int c0 = 0; c0 < ncol; c0 += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (c0 + k < ncol) v[k] = __ldcg(src + (size_t)((c0 + k) * s.U + u) * REC4);
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (c0 + k < ncol) add4(sum, v[k]);
+    }
     if (s.m > 0) {
       const int r_lo = trailing_cta_of((long long)u * s.m, ttot, s.R);
       const int r_hi = trailing_cta_of((long long)(u + 1) * s.m - 1, ttot, s.R);
-      for (int r = r_lo; r <= r_hi; ++r) sum += __ldcg(src + (size_t)(s.P * s.U + r + u) * (C::G * E));
+      for (int r0 = r_lo; r0 <= r_hi; r0 += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (r0 + k <= r_hi) v[k] = __ldcg(src + (size_t)(s.P * s.U + r0 + k + u) * REC4);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (r0 + k <= r_hi) add4(sum, v[k]);
+      }
     }
-    p.state[idx] = sum;
+    state4[idx] = sum;
   }
 }
 
@@ -269,29 +297,47 @@ __device__ __forceinline__ void build_s_operand(uint8_t* s_op, const float* __re
   using C = Cfg<D>;
   constexpr int CPR = D / 8;       // 16-byte chunks per state row
   constexpr int ROWS = D + 1;
-  for (int idx = part; idx < C::G * ROWS * CPR; idx += nparts) {
-    const int g = idx / (ROWS * CPR);
-    const int rem = idx - g * ROWS * CPR;
-    const int j = rem / CPR, c = rem % CPR;
-    const int h = hg * C::G + g;
-    float x[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    if (h < H) {
-      const float4* src = reinterpret_cast<const float4*>(state + ((size_t)(b * H + h) * ROWS + j) * D + c * 8);
-      const float4 a = __ldcg(src), bq = __ldcg(src + 1);
-      x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = bq.x; x[5] = bq.y; x[6] = bq.z; x[7] = bq.w;
-    }
-    uint32_t hi[4], lo[4];
+  constexpr int TOTAL = C::G * ROWS * CPR;
+  constexpr int BATCH = 4;         // chunks whose loads are in flight together
+  for (int base = part; base < TOTAL; base += BATCH * nparts) {
+    float4 lo4[BATCH], hi4[BATCH];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
-      hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-      lo[e] = pack_bf16x2(x[2 * e] - __bfloat162float(h0), x[2 * e + 1] - __bfloat162float(h1));
+    for (int k = 0; k < BATCH; ++k) {
+      const int idx = base + k * nparts;
+      lo4[k] = hi4[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (idx < TOTAL) {
+        const int g = idx / (ROWS * CPR);
+        const int rem = idx - g * ROWS * CPR;
+        const int j = rem / CPR, c = rem % CPR;
+        const int h = hg * C::G + g;
+        if (h < H) {
+          const float4* src = reinterpret_cast<const float4*>(state + ((size_t)(b * H + h) * ROWS + j) * D + c * 8);
+          lo4[k] = __ldcg(src);
+          hi4[k] = __ldcg(src + 1);
+        }
+      }
     }
-    const int jrow = j < D ? g * D + j : C::ZROW + g;  // operand row: value feature, or the head's z row
-    const int i0 = g * D + c * 8;                      // first key feature of this chunk
-    const int off = (i0 >> 6) * C::SBOX_BYTES + jrow * kRowBytes + ((((i0 & 63) >> 3) ^ (jrow & 7)) << 4);
-    *reinterpret_cast<uint4*>(s_op + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    *reinterpret_cast<uint4*>(s_op + 2 * C::SBOX_BYTES + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+#pragma unroll
+    for (int k = 0; k < BATCH; ++k) {
+      const int idx = base + k * nparts;
+      if (idx >= TOTAL) break;
+      const int g = idx / (ROWS * CPR);
+      const int rem = idx - g * ROWS * CPR;
+      const int j = rem / CPR, c = rem % CPR;
+      const float x[8] = {lo4[k].x, lo4[k].y, lo4[k].z, lo4[k].w, hi4[k].x, hi4[k].y, hi4[k].z, hi4[k].w};
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
+        hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+        lo[e] = pack_bf16x2(x[2 * e] - __bfloat162float(h0), x[2 * e + 1] - __bfloat162float(h1));
+      }
+      const int jrow = j < D ? g * D + j : C::ZROW + g;  // operand row: value feature, or the head's z row
+      const int i0 = g * D + c * 8;                      // first key feature of this chunk
+      const int off = (i0 >> 6) * C::SBOX_BYTES + jrow * kRowBytes + ((((i0 & 63) >> 3) ^ (jrow & 7)) << 4);
+      *reinterpret_cast<uint4*>(s_op + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(s_op + 2 * C::SBOX_BYTES + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
   }
 }
 
@@ -409,7 +455,20 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         tma_load_4d(st + C::KOFF + kBox, &map_k, &a_full[s], c0, c1, t.tile() * kTileState, b);
         tma_load_4d(st + kBox, &map_v, &a_full[s], c0, c1, t.tile() * kTileState, b);
       }
-      // the stages are free once every MMA of this pass is complete: start on the Q tiles now
+      // Q does not depend on the state: ask for the first tiles now (into L2; requesting tiles further
+      // ahead than this, in either pass, measured slower), and fill the slots as soon as every MMA of this
+      // pass is complete (the stages are free then)
+      {
+        TileWalk t(wc);
+        for (int i = 0; i < NSC && !t.done(); ++i, t.next()) {
+          const int u = t.unit(), b = u / p.HG, hg = u % p.HG;
+          int c0, c1;
+          box_coords<D>(0, hg, c0, c1);
+          tma_prefetch_4d(&map_q, c0, c1, t.tile() * kTileApply, b);
+          box_coords<D>(1, hg, c0, c1);
+          tma_prefetch_4d(&map_q, c0, c1, t.tile() * kTileApply, b);
+        }
+      }
       if (wc.f1 > wc.f0 && mbar_wait(a_done, 0, abort_flag)) {
         while (!cw.done() && c_it < (uint32_t)NSC)
           if (!load_q_tile()) break;
@@ -449,7 +508,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       const int s = it % NSA;
       if (!mbar_wait(&a_full[s], (it / NSA) & 1, abort_flag)) break;
       uint8_t* st = smem + s * STAGE;
-      relu_pass<C::FEAT>(st + C::KOFF, 2 * kBox / 16, kBox / 16, tr);
+      relu_pass<C::FEAT, kTileState>(st + C::KOFF, st + C::KOFF + kBox, tr);
       if (!C::ONES_BOX && tr < kTileState) {
         // value column 112 := 1 (logical chunk 6 of the second V box, element 0), so z is accumulator column 112
         *reinterpret_cast<uint16_t*>(st + kBox + tr * kRowBytes + ((6 ^ (tr & 7)) << 4)) = 0x3F80u;
@@ -570,7 +629,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         ++seg;
       }
       if (!mbar_wait(&c_full[s], (it / NSC) & 1, abort_flag)) break;
-      relu_pass<C::FEAT>(slots + s * SLOT, SLOT / 16, HALF / 16, tr);
+      relu_pass<C::FEAT, kTileApply>(slots + s * SLOT, slots + s * SLOT + HALF, tr);
       fence_proxy_async_smem();
       mbar_arrive(&c_ready[s]);
     }
