@@ -72,7 +72,9 @@ struct Cfg {
   static constexpr int STAGE_BYTES = (ONES_BOX ? 5 : 4) * kBox;        // V0 V1 [ONES] K0 K1
   static constexpr int KOFF = (ONES_BOX ? 3 : 2) * kBox;               // K boxes within a stage
   static constexpr int DATA_BYTES = S_BYTES + APPLY_SLOTS * SLOT_BYTES;
-  static constexpr int STATE_STAGES = DATA_BYTES / STAGE_BYTES;        // the state pass uses the whole data area
+  // The data area would hold up to seven stages, but four measured fastest: with more bytes in flight
+  // per SM the memory system's queues grow and the SMs' shares of the bandwidth drift apart.
+  static constexpr int STATE_STAGES = DATA_BYTES / STAGE_BYTES < 4 ? DATA_BYTES / STAGE_BYTES : 4;
   static constexpr int BAR_BYTES = 1024;
   static constexpr size_t SMEM = 1024 + DATA_BYTES + BAR_BYTES;
 };
