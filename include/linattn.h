@@ -75,7 +75,9 @@ typedef enum linattn_status {
   LINATTN_ERR_WORKSPACE_TOO_SMALL = -4,
   LINATTN_ERR_CUDA = -5,               /* a CUDA runtime/driver call failed, or no sm_100 device */
   LINATTN_ERR_TIMEOUT = -6,            /* a bounded device-side wait expired */
-  LINATTN_ERR_BAD_HANDLE = -7          /* cache handle is null, destroyed or corrupt */
+  LINATTN_ERR_BAD_HANDLE = -7,         /* cache handle is null, destroyed or corrupt */
+  LINATTN_ERR_SCRATCH_LIMIT = -8       /* problem needs more scratch than the built-in array of
+                                          linattn_state_static_scratch holds */
 } linattn_status;
 
 /* Problem descriptor: plain data, filled by the caller, copied by the library. */
@@ -116,6 +118,32 @@ LINATTN_API int linattn_forward(const linattn_desc* desc, int64_t N, const void*
  * Deterministic: split-N partials are summed in a fixed order, so repeated calls give identical bits. */
 LINATTN_API int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void* v, float* state,
                   void* workspace, size_t workspace_bytes, void* stream);
+
+/* linattn_state for callers that cannot provide a workspace.  (The paper has no counterpart: this
+ * is a convenience of this library.)
+ *
+ * Some callers may not allocate device memory at the point where they need the state: code running
+ * inside a memory-budgeted serving loop whose pools are fixed at start-up, a plug-in that is handed
+ * tensors but no allocator, or a host thread that must not take the allocator's lock because
+ * cudaMalloc may synchronise the whole device.  For them the split-N scratch of the state pass lives
+ * in an array compiled into the library instead of a caller-provided workspace.  This function
+ * calls no cudaMalloc / cudaFree and no allocating library routine; the caller still passes the
+ * inputs k, v and the output `state` (same meaning, layout and alignment rules as linattn_state).
+ *
+ *  - Limit: the scratch the call needs (what linattn_workspace_bytes reports, minus the trailing
+ *    state slot) must fit in LINATTN_STATIC_SCRATCH_BYTES (16 MiB; every GPU on which this library
+ *    is used holds that much device memory until the process exits).  That covers, for example,
+ *    B*H <= 20 heads of dimension 112 at any N.  Larger problems return
+ *    LINATTN_ERR_SCRATCH_LIMIT and launch nothing.
+ *  - The first call on each device looks the array's device address up (one runtime call, with
+ *    that device current); make that first call outside any stream capture.
+ *  - Every call on a device shares the one array, which still holds the previous call's contents:
+ *    the control block at its start is cleared on `stream` before every launch, and the partial
+ *    records are fully rewritten before they are read.  Two calls that overlap on the GPU (different
+ *    streams, or threads racing on one device) would corrupt each other: order them. */
+#define LINATTN_STATIC_SCRATCH_BYTES (16u << 20)
+LINATTN_API int linattn_state_static_scratch(const linattn_desc* desc, int64_t N, const void* k, const void* v,
+                                             float* state, void* stream);
 
 /* The apply half of Eq. 2 alone: o_n = phi(q_n) S / (phi(q_n) . z + eps) for a given state.
  * workspace: only its control block is used (LINATTN_WORKSPACE_CTRL_BYTES suffice). */

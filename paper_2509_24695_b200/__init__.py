@@ -18,7 +18,7 @@ import os
 
 __all__ = [
     "LinAttnError", "library_path", "load_library", "state_bytes", "workspace_bytes", "new_workspace",
-    "linattn_forward", "linattn_state", "linattn_apply", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
+    "linattn_forward", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
 ]
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -71,6 +71,7 @@ def load_library(path: str | None = None):
         "linattn_forward": ([dp, i64, vp, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
         "linattn_state": ([dp, i64, vp, vp, vp, vp, sz, vp], ctypes.c_int),
         "linattn_apply": ([dp, i64, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
+        "linattn_state_static_scratch": ([dp, i64, vp, vp, vp, vp], ctypes.c_int),
         "linattn_forward_host_bytes": ([dp, i64, szp], ctypes.c_int),
         "linattn_forward_host": ([dp, i64, vp, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
         "linattn_kernel_launches": ([], ctypes.c_uint64),
@@ -223,6 +224,28 @@ def linattn_state(k, v, out=None, workspace=None):
     _check(lib.linattn_state(ctypes.byref(desc), N, _ptr(k), _ptr(v), _ptr(st), _ptr(ws), ws.numel(), _stream(k)),
            "linattn_state")
     return st
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def linattn_state_static_scratch(k, v, out):
+    """``linattn_state`` without a workspace: for callers that must not allocate device memory.
+
+    The split-N scratch is an array built into the library (``STATIC_SCRATCH_BYTES``, shared by all
+    calls on a device), so this wrapper allocates nothing either: ``out`` (float32 ``[B, H, d+1, d]``)
+    is required.  Problems whose scratch does not fit raise ``LinAttnError`` with status -8.  Calls
+    on one device must not overlap on the GPU; make the first call outside stream capture.
+    """
+    torch = _torch()
+    lib = load_library()
+    desc = _desc_of(k, v)
+    B, N, H, d = k.shape
+    if tuple(out.shape) != (B, H, d + 1, d) or out.dtype != torch.float32 or not out.is_contiguous():
+        raise ValueError("out must be a contiguous float32 [B, H, d+1, d] tensor")
+    _check(lib.linattn_state_static_scratch(ctypes.byref(desc), N, _ptr(k), _ptr(v), _ptr(out), _stream(k)),
+           "linattn_state_static_scratch")
+    return out
 
 
 def linattn_apply(q, state, eps: float = 1e-6, out=None, workspace=None):

@@ -86,6 +86,26 @@ int run_passes(const Problem& p, const void* k, const void* v, const void* q, vo
 
 }  // namespace
 
+// Scratch of linattn_state_static_scratch: part of the library image, so no call has to allocate it.
+// In host code this name is only a handle for the runtime; the device address comes from
+// cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[LINATTN_STATIC_SCRATCH_BYTES];
+
+static void* static_scratch_address() {
+  static void* cached[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cached[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    cached[dev] = ptr;
+  }
+  return cached[dev];
+}
+
 struct blocklin_cache {
   uint32_t magic;
   linattn_desc desc;
@@ -127,6 +147,7 @@ const char* linattn_status_string(int status) {
     case LINATTN_ERR_CUDA: return "CUDA call failed";
     case LINATTN_ERR_TIMEOUT: return "bounded device-side wait expired";
     case LINATTN_ERR_BAD_HANDLE: return "bad cache handle";
+    case LINATTN_ERR_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of linattn_state_static_scratch";
     default: return "unknown status";
   }
 }
@@ -175,6 +196,25 @@ int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void
   if (workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
   if (N == 0) return cuda_status(cudaMemsetAsync(state, 0, state_bytes_of(p), (cudaStream_t)stream));  // empty sum
   return run_passes(p, k, v, nullptr, nullptr, state, false, 0.f, workspace, (cudaStream_t)stream);
+}
+
+int linattn_state_static_scratch(const linattn_desc* desc, int64_t N, const void* k, const void* v, float* state,
+                                 void* stream) {
+  Problem p;
+  int st = resolve(desc, N, &p);
+  if (st != LINATTN_OK) return st;
+  if (!state) return LINATTN_ERR_INVALID_ARG;
+  if (N > 0 && (!k || !v)) return LINATTN_ERR_INVALID_ARG;
+  if ((st = check_alignment(p, k, v, state, nullptr)) != LINATTN_OK) return st;
+  // control block + split-N partials; the state slot that linattn_forward keeps behind them is not needed
+  if (state_slot_offset(p) > sizeof(g_static_scratch)) return LINATTN_ERR_SCRATCH_LIMIT;
+  void* scratch = static_scratch_address();
+  if (!scratch) return LINATTN_ERR_CUDA;
+  if (N == 0) return cuda_status(cudaMemsetAsync(state, 0, state_bytes_of(p), (cudaStream_t)stream));  // empty sum
+  // the array keeps the last call's contents: the barrier word and the status word must start at zero
+  if (cudaMemsetAsync(scratch, 0, LINATTN_WORKSPACE_CTRL_BYTES, (cudaStream_t)stream) != cudaSuccess)
+    return LINATTN_ERR_CUDA;
+  return run_passes(p, k, v, nullptr, nullptr, state, false, 0.f, scratch, (cudaStream_t)stream);
 }
 
 int linattn_apply(const linattn_desc* desc, int64_t N, const void* q, const float* state, void* o, float eps,
