@@ -263,28 +263,27 @@ __device__ void reduce_slice(const FusedParams& p) {
     const int u = b * p.HG + h / C::G, g = h % C::G;
     const float4* src = reinterpret_cast<const float4*>(p.partials) + (size_t)g * E4 + e;
     float4 sum = p.accumulate ? __ldcg(state4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
-    // the loads of a batch are independent and issued together; the adds keep the fixed order
-    for (int c0 = 0; c0 < ncol; c0 += 8) {
-      float4 v[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k)
-        if (c0 + k < ncol) v[k] = __ldcg(src + (size_t)((c0 + k) * s.U + u) * REC4);
-#pragma unroll
-      for (int k = 0; k < 8; ++k)
-        if (c0 + k < ncol) add4(sum, v[k]);
-    }
+    // every record of the unit, column CTAs first, then the trailing CTAs; the loads of a batch are
+    // independent and issued together, the adds keep that fixed order
+    int r_lo = 0, ntrail = 0;
     if (s.m > 0) {
-      const int r_lo = trailing_cta_of((long long)u * s.m, ttot, s.R);
-      const int r_hi = trailing_cta_of((long long)(u + 1) * s.m - 1, ttot, s.R);
-      for (int r0 = r_lo; r0 <= r_hi; r0 += 4) {
-        float4 v[4];
+      r_lo = trailing_cta_of((long long)u * s.m, ttot, s.R);
+      ntrail = trailing_cta_of((long long)(u + 1) * s.m - 1, ttot, s.R) - r_lo + 1;
+    }
+    const int nrec = ncol + ntrail;
+    for (int k0 = 0; k0 < nrec; k0 += 12) {
+      float4 v[12];
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (r0 + k <= r_hi) v[k] = __ldcg(src + (size_t)(s.P * s.U + r0 + k + u) * REC4);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (r0 + k <= r_hi) add4(sum, v[k]);
+      for (int k = 0; k < 12; ++k) {
+        const int kk = k0 + k;
+        if (kk < nrec) {
+          const int rec = kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u;
+          v[k] = __ldcg(src + (size_t)rec * REC4);
+        }
       }
+#pragma unroll
+      for (int k = 0; k < 12; ++k)
+        if (k0 + k < nrec) add4(sum, v[k]);
     }
     state4[idx] = sum;
   }
@@ -300,7 +299,7 @@ __device__ __forceinline__ void build_s_operand(uint8_t* s_op, const float* __re
   constexpr int CPR = D / 8;       // 16-byte chunks per state row
   constexpr int ROWS = D + 1;
   constexpr int TOTAL = C::G * ROWS * CPR;
-  constexpr int BATCH = 4;         // chunks whose loads are in flight together
+  constexpr int BATCH = 7;         // chunks whose loads are in flight together (all of a thread's share at d = 112)
   for (int base = part; base < TOTAL; base += BATCH * nparts) {
     float4 lo4[BATCH], hi4[BATCH];
 #pragma unroll
