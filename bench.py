@@ -172,6 +172,20 @@ def run_reference(args):
     }))
 
 
+def max_over_ranks(torch, dist, ms: float, device) -> float:
+    """A multi-rank time is the slowest rank's: all-reduce MAX (NCCL on GPUs, gloo in the CPU tests)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, units_per_rank: int, ms_per_step: float) -> float:
+    """Weak scaling: every rank processes `units_per_rank` tokens*heads per step on its own shard."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 def time_loop(torch, fn, steps, sync_ranks=None):
     """CUDA-event time of `steps` calls of fn(i) on the current stream, in ms."""
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -248,12 +262,9 @@ def main():
         step(0)
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    if dist:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(torch, dist, ms, dev)
     ms_per_step = ms / K
-    value = world * units / (ms_per_step * 1e-3)
+    value = whole_job_value(world, units, ms_per_step)
 
     # per-kernel split: state pass and apply pass timed live, each as its own entry point
     state_buf = la.linattn_state(sets[0][1], sets[0][2], workspace=ws)
@@ -286,11 +297,8 @@ def main():
         for _ in range(2):
             hf(qp, kp, vp, op, w.eps)
         ms_e2e = time_loop(torch, lambda i: hf(qp, kp, vp, op, w.eps), k_e2e, sync_ranks)
-        if dist:
-            t = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e = {"value": world * units / (ms_e2e / k_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": hf.h2d_bytes,
+        ms_e2e = max_over_ranks(torch, dist, ms_e2e, dev)
+        e2e = {"value": whole_job_value(world, units, ms_e2e / k_e2e), "unit": UNIT, "h2d_bytes_per_step": hf.h2d_bytes,
                "d2h_bytes_per_step": hf.d2h_bytes, "steps": k_e2e, "ms_per_step": ms_e2e / k_e2e}
         assert float(op.float().abs().sum()) > 0.0
 

@@ -63,6 +63,11 @@ struct Cfg {
   static constexpr bool ONES_BOX = D != 112;
   static constexpr int NSTATE = ONES_BOX ? 144 : 128;        // state MMA N
   static constexpr int ZCOL = ONES_BOX ? 128 : 112;          // state accumulator column that holds z
+  // The tensor core truncates when it adds into the fp32 accumulator, so a long chain of updates drifts
+  // (about 2^-24 relative per update).  The state pass therefore deals its MMAs round-robin to several
+  // accumulators, which the epilogue adds up (round to nearest) once per segment: shorter chains.
+  static constexpr int STATE_ACCS = ONES_BOX ? 3 : 4;
+  static constexpr int STATE_ACC_STRIDE = ONES_BOX ? 160 : 128;   // TMEM columns between them
   static constexpr int BOX_D = 64;                           // TMA box: features ...
   static constexpr int BOX_H = 1;                            // ... x heads
   static constexpr int SBOX_BYTES = NAPPLY * kRowBytes;      // one 64-feature K box of the S operand
@@ -364,8 +369,8 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   uint64_t* a_full = bars;                 // TMA landed
   uint64_t* a_ready = a_full + NSA;        // ReLU pass done
   uint64_t* a_empty = a_ready + NSA;       // MMAs that read the stage are complete
-  uint64_t* a_tfull = a_empty + NSA;       // [2] accumulator complete
-  uint64_t* a_tempty = a_tfull + 2;        // [2] accumulator drained by the epilogue
+  uint64_t* a_tfull = a_empty + NSA;       // the segment's accumulators are complete
+  uint64_t* a_tempty = a_tfull + 2;        // ... and drained by the epilogue
   uint64_t* a_done = a_tempty + 2;         // every MMA of the state pass is complete: stages are free
   // apply pass
   uint64_t* c_full = a_done + 1;           // Q tile landed
@@ -386,7 +391,8 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_ready[s], 128); mbar_init(&a_empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&a_tfull[b], 1); mbar_init(&a_tempty[b], 128); }
+    mbar_init(a_tfull, 1);
+    mbar_init(a_tempty, 128);
     mbar_init(a_done, 1);
     for (int s = 0; s < NSC; ++s) {
       mbar_init(&c_full[s], 1); mbar_init(&c_ready[s], 128); mbar_init(&c_empty[s], 1); mbar_init(&c_staged[s], 128);
@@ -478,26 +484,25 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      uint32_t it = 0, seg = 0;
+      uint32_t it = 0, seg = 0, n_mma = 0;
       bool ok = true;
       for (TileWalk t(wa); !t.done() && ok; t.next(), ++it) {
         const int s = it % NSA;
         const bool seg_first = t.seg_first();
-        const uint32_t acc = seg & 1;
-        if (seg_first) ok = mbar_wait(&a_tempty[acc], ((seg >> 1) & 1) ^ 1, abort_flag);
+        if (seg_first) { ok = mbar_wait(a_tempty, (seg & 1) ^ 1, abort_flag); n_mma = 0; }
         if (ok) ok = mbar_wait(&a_ready[s], (it / NSA) & 1, abort_flag);
         if (!ok) break;
         tcgen05_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * kAccStride;
         const uint32_t st = smem_u32(smem + s * STAGE);
 #pragma unroll
-        for (int kk = 0; kk < kTileState / 16; ++kk) {
+        for (int kk = 0; kk < kTileState / 16; ++kk, ++n_mma) {
           const uint64_t a = make_smem_desc_sw128(st + C::KOFF + kk * 2048, kBox, 1024);  // phi(K)^T, MN-major
           const uint64_t bq = make_smem_desc_sw128(st + kk * 2048, kBox, 1024);           // [V | 1], MN-major
-          umma_bf16(d_tmem, a, bq, IDESC_A, (seg_first && kk == 0) ? 0u : 1u);
+          const uint32_t d_tmem = tmem_base + (n_mma % C::STATE_ACCS) * C::STATE_ACC_STRIDE;
+          umma_bf16(d_tmem, a, bq, IDESC_A, n_mma < (uint32_t)C::STATE_ACCS ? 0u : 1u);  // first use of each: overwrite
         }
         umma_commit(&a_empty[s]);
-        if (t.seg_last()) { umma_commit(&a_tfull[acc]); ++seg; }
+        if (t.seg_last()) { umma_commit(a_tfull); ++seg; }
       }
       if (it > 0) umma_commit(a_done); else mbar_arrive(a_done);
     }
@@ -525,8 +530,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     uint32_t seg = 0;
     for (TileWalk t(wa); !t.done(); t.next()) {
       if (!t.seg_last()) continue;
-      const uint32_t acc = seg & 1;
-      bool ok = mbar_wait(&a_tfull[acc], (seg >> 1) & 1, abort_flag);
+      bool ok = mbar_wait(a_tfull, seg & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
@@ -535,30 +539,49 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       const bool live = i < C::FEAT && h < p.H;
       // record of this (CTA, unit) segment: G consecutive head-states in the library's layout
       float* out = p.partials + ((size_t)t.record() * C::G + g) * ((size_t)(D + 1) * D);
-      const uint32_t trow = tmem_base + acc * kAccStride + ((uint32_t)(wq * 32) << 16);
+      const uint32_t trow = tmem_base + ((uint32_t)(wq * 32) << 16);
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
-        uint32_t r[32];
-        tmem_ld_x32(trow + cc * 32, r);
-        tmem_ld_wait();
+        // the accumulators are added in a fixed order (round to nearest)
+        float sum[32];
+        {
+          uint32_t r[32];
+          tmem_ld_x32(trow + cc * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int x = 0; x < 32; ++x) sum[x] = __uint_as_float(r[x]);
+        }
+#pragma unroll 1
+        for (int a = 1; a < C::STATE_ACCS; ++a) {
+          uint32_t r[32];
+          tmem_ld_x32(trow + a * C::STATE_ACC_STRIDE + cc * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int x = 0; x < 32; ++x) sum[x] += __uint_as_float(r[x]);
+        }
         if (live) {
 #pragma unroll
           for (int x = 0; x < 32; ++x) {
             const int j = cc * 32 + x;             // value feature within the group
             const int jl = j - g * D;
-            if (jl >= 0 && jl < D) out[(size_t)jl * D + il] = __uint_as_float(r[x]);
-            if (!C::ONES_BOX && j == C::ZCOL) out[(size_t)D * D + il] = __uint_as_float(r[x]);
+            if (jl >= 0 && jl < D) out[(size_t)jl * D + il] = sum[x];
+            if (!C::ONES_BOX && j == C::ZCOL) out[(size_t)D * D + il] = sum[x];
           }
         }
       }
       if (C::ONES_BOX) {
-        uint32_t zr[4];
-        tmem_ld_x4(trow + C::ZCOL, zr);
-        tmem_ld_wait();
-        if (live) out[(size_t)D * D + il] = __uint_as_float(zr[0]);
+        float zsum = 0.f;
+#pragma unroll 1
+        for (int a = 0; a < C::STATE_ACCS; ++a) {
+          uint32_t zr[4];
+          tmem_ld_x4(trow + a * C::STATE_ACC_STRIDE + C::ZCOL, zr);
+          tmem_ld_wait();
+          zsum = a == 0 ? __uint_as_float(zr[0]) : zsum + __uint_as_float(zr[0]);
+        }
+        if (live) out[(size_t)D * D + il] = zsum;
       }
       tcgen05_fence_before();
-      mbar_arrive(&a_tempty[acc]);
+      mbar_arrive(a_tempty);
       ++seg;
     }
   }

@@ -1,0 +1,116 @@
+"""GPU parity at the full workload sizes, in the launch configuration the benchmark times.
+
+The oracle cannot produce every output row of a 75 600-token layer in seconds, but it can produce the
+state exactly (one pass over K, V) and then any sampled row one by one; so at full size the CUDA path is
+checked on (i) the whole fp32 state against the oracle's fp64 state and (ii) sampled output rows (ends,
+tile edges, seeded random picks) against the oracle's apply of ITS OWN state to those rows.
+"""
+import numpy as np
+import pytest
+
+from paper_2509_24695_b200 import synth
+from parity_util import assert_parity_bf16, assert_state_close, sample_rows, to_dev, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def la():
+    import torch
+
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    import paper_2509_24695_b200 as la
+
+    la.load_library()
+    return la
+
+
+def _check_bidirectional(la, orc, w, n_rows=96):
+    import torch
+
+    q, k, v = synth.qkv(w)
+    qd, kd, vd = to_dev(q), to_dev(k), to_dev(v)
+    ws = la.new_workspace(qd)
+    o = la.linattn_forward(qd, kd, vd, w.eps, workspace=ws)      # the call bench.py times
+    st = la.linattn_state(kd, vd, workspace=ws)
+    assert la.workspace_status(ws) == 0
+    S, z = orc.state(k, v)
+    assert_state_close(to_f64(st), S, z, 1e-5, f"{w.name} state")
+    rows = sample_rows(w.N, n_rows, w.seed)
+    ref = orc.apply_rows(q, S, z, w.eps, rows)
+    got = to_f64(o[:, torch.from_numpy(rows).cuda()])
+    assert_parity_bf16(got, ref, f"{w.name} sampled rows")
+    # property that holds at any size: no row is left unwritten / non-finite
+    assert torch.isfinite(o.float()).all()
+    assert (o.float().abs().amax(dim=(0, 2, 3)) > 0).all()
+
+
+def test_480p_layer(la, orc):
+    _check_bidirectional(la, orc, synth.P480)
+
+
+def test_720p_layer(la, orc):
+    _check_bidirectional(la, orc, synth.P720)
+
+
+@pytest.mark.parametrize("d", [32, 64, 128])
+def test_720p_head_dim_sweep(la, orc, d):
+    _check_bidirectional(la, orc, synth.p720_sweep(d), n_rows=48)
+
+
+def test_480p_block_causal_seven_steps(la, orc):
+    """Config 4 at full size: 7 steps of 4680 tokens against the oracle's block-wise prefix states."""
+    import torch
+
+    w = synth.AR480
+    cache = la.BlockLinCache(w.B, w.H, w.d, torch.bfloat16, "cuda", max_T_b=w.T_b, eps=w.eps)
+    S, z = orc.new_cache(w.B, w.H, w.d)
+    rows = sample_rows(w.T_b, 40, w.seed)
+    outs = []
+    for b in range(w.n_blocks):
+        q, k, v = synth.qkv_block(w, b)
+        o = cache.step(to_dev(q), to_dev(k), to_dev(v))
+        outs.append(o)
+        Sb, zb = orc.state(k, v)
+        S += Sb; z += zb                      # Eq. 3: the cache is the running sum of block states
+        ref = orc.apply_rows(q, S, z, w.eps, rows)
+        assert_parity_bf16(to_f64(o[:, torch.from_numpy(rows).cuda()]), ref, f"{w.name} block {b}")
+        assert cache.info()["state_bytes"] == w.B * w.H * (w.d * w.d + w.d) * 4
+    assert_state_close(to_f64(cache.state), S, z, 1e-5, "cache after 7 blocks")
+    # one prefill call over the whole sequence gives the same bits and the same cache
+    final = cache.state.clone()
+    cache.reset()
+    q, k, v = synth.qkv(w)
+    o_pre = cache.prefill(to_dev(q), to_dev(k), to_dev(v), w.n_blocks)
+    assert torch.equal(o_pre, torch.cat(outs, dim=1))
+    assert torch.equal(cache.state, final)
+    assert la.workspace_status(cache.workspace) == 0
+
+
+def test_720p_stream_eighty_steps(la, orc):
+    """Config 5's shape (B=2, 10800 tokens per block, 80 steps).  Three distinct seeded blocks are cycled,
+    so the oracle's cache after any number of steps is a count-weighted sum of three block states; the
+    fp32 cache is compared with it after steps 1, 40 and 80, and the last step's sampled rows too."""
+    import torch
+
+    w = synth.STREAM720
+    blocks = [synth.qkv_block(w, b) for b in range(3)]
+    dev = [tuple(to_dev(x) for x in blk) for blk in blocks]
+    states = [orc.state(k, v) for (_, k, v) in blocks]
+    cache = la.BlockLinCache(w.B, w.H, w.d, torch.bfloat16, "cuda", max_T_b=w.T_b, eps=w.eps)
+    bytes0 = cache.info()["state_bytes"]
+    assert bytes0 == w.B * w.H * (w.d * w.d + w.d) * 4 == 2024960
+    out = torch.empty_like(dev[0][0])
+    for step in range(1, w.n_blocks + 1):
+        cache.step(*dev[(step - 1) % 3], out=out)
+        assert cache.info() == {"blocks_seen": step, "tokens_seen": step * w.T_b, "state_bytes": bytes0}
+        if step in (1, 40, 80):
+            counts = [(step + 2 - i) // 3 for i in range(3)]
+            S = sum(c * s[0] for c, s in zip(counts, states))
+            z = sum(c * s[1] for c, s in zip(counts, states))
+            assert_state_close(to_f64(cache.state), S, z, 1e-5, f"cache after {step} blocks")
+    rows = sample_rows(w.T_b, 40, w.seed)
+    q_last = blocks[(w.n_blocks - 1) % 3][0]
+    ref = orc.apply_rows(q_last, S, z, w.eps, rows)
+    assert_parity_bf16(to_f64(out[:, torch.from_numpy(rows).cuda()]), ref, "last step sampled rows")
+    assert la.workspace_status(cache.workspace) == 0
