@@ -124,17 +124,29 @@ __host__ __device__ inline Work work_of(const Sched& s, int j) {
   return w;
 }
 
-inline Sched make_sched(int U, long long tpu, int max_ctas) {
+// `seg_cost`: what starting one more unit segment costs a CTA, in tiles (drain of the accumulators /
+// rebuild of the S operand).  Trailing CTAs cross several units, so the columns are made a little longer
+// until the trailing CTAs' tiles plus their segment starts fit into a column's time.
+inline Sched make_sched(int U, long long tpu, int max_ctas, int seg_cost) {
   Sched s;
   const long long total = (long long)U * tpu;
   s.U = U; s.tpu = (int)tpu;
   s.grid = (int)(total < max_ctas ? total : max_ctas);
   if (s.grid < 1) s.grid = 1;
   s.P = s.grid / U;
-  s.Lc = (int)((total + s.grid - 1) / s.grid);
+  s.R = s.grid - s.P * U;
+  const int lc0 = (int)((total + s.grid - 1) / s.grid);
+  s.Lc = lc0;
+  if (s.P > 0 && s.R > 0) {
+    for (int lc = lc0; lc < lc0 + 8; ++lc) {
+      const long long m = (long long)s.P * lc >= tpu ? 0 : tpu - (long long)s.P * lc;
+      const long long tiles = (U * m + s.R - 1) / s.R;
+      const long long segs = m > 0 ? (tiles + m - 1) / m + 1 : 0;
+      if (tiles + segs * seg_cost <= lc) { s.Lc = lc; break; }
+    }
+  }
   const long long covered = (long long)s.P * s.Lc;
   s.m = covered >= tpu ? 0 : (int)(tpu - covered);
-  s.R = s.grid - s.P * U;
   return s;
 }
 
@@ -812,8 +824,8 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   FusedParams fp{};
   fp.B = p.B; fp.H = p.H; fp.HG = (p.H + C::G - 1) / C::G;
   const int U = p.B * fp.HG;
-  fp.sa = make_sched(U, (p.N + kTileState - 1) / kTileState, sms);
-  fp.sc = make_sched(U, (p.N + kTileApply - 1) / kTileApply, sms);
+  fp.sa = make_sched(U, (p.N + kTileState - 1) / kTileState, sms, 2);
+  fp.sc = make_sched(U, (p.N + kTileApply - 1) / kTileApply, sms, 2);
   fp.do_state = do_state; fp.do_apply = do_apply; fp.accumulate = c.accumulate ? 1 : 0;
   fp.state = c.state;
   fp.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + LINATTN_WORKSPACE_CTRL_BYTES);
