@@ -188,6 +188,13 @@ LINATTN_API int blocklin_cache_reset(blocklin_cache* cache, void* stream);
 LINATTN_API int blocklin_step(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
                   void* o_blk, void* stream);
 
+/* The denoising steps of Algorithm 1 ("x0 <- G(x; t_j, KV)" for t_j > 0): the block's queries see the
+ * cache plus the block's own (S_blk, z_blk), exactly as in blocklin_step, but the cache is only read:
+ * nothing is committed, blocks_seen does not change.  The clean block is committed afterwards with
+ * blocklin_step (with q_blk = o_blk = NULL to commit without producing outputs). */
+LINATTN_API int blocklin_peek(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
+                  void* o_blk, void* stream);
+
 /* n_blocks consecutive blocks of T_b tokens in one call over [B, n_blocks*T_b, H, d] tensors;
  * result and final cache equal n_blocks calls of blocklin_step.  q and o may both be NULL. */
 LINATTN_API int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,

@@ -79,6 +79,7 @@ def load_library(path: str | None = None):
         "blocklin_cache_init": ([ctypes.POINTER(vp), dp, f32, vp, sz, vp, sz, vp], ctypes.c_int),
         "blocklin_cache_reset": ([vp, vp], ctypes.c_int),
         "blocklin_step": ([vp, i64, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_peek": ([vp, i64, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_prefill": ([vp, i64, i64, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_cache_info": ([vp, ctypes.POINTER(i64), ctypes.POINTER(i64), szp], ctypes.c_int),
         "blocklin_cache_destroy": ([vp], ctypes.c_int),
@@ -312,6 +313,16 @@ class BlockLinCache:
         self._check_layout(k)
         _check(self._lib.blocklin_step(self._handle, k.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o), _stream(k)),
                "blocklin_step")
+        return o
+
+    def peek(self, q, k, v, out=None):
+        """Output of the block against cache + state(block) without committing (Algorithm 1's denoising steps)."""
+        torch = _torch()
+        o = torch.empty_like(q) if out is None else out
+        _desc_of(q, k, v, o)
+        self._check_layout(k)
+        _check(self._lib.blocklin_peek(self._handle, k.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o), _stream(k)),
+               "blocklin_peek")
         return o
 
     def prefill(self, q, k, v, n_blocks: int, out=None):

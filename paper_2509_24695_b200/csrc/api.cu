@@ -68,13 +68,18 @@ inline float* partials_of(void* workspace) {
 
 int cuda_status(cudaError_t e) { return e == cudaSuccess ? LINATTN_OK : LINATTN_ERR_CUDA; }
 
-// state_out = (accumulate ? state_out : 0) + state(k, v), then (q non-null) o = apply(q, state_out).
-// On the tensor-core path both halves run in one launch.
+// state = (accumulate ? base : 0) + state(k, v), then (q non-null) o = apply(q, state).  `base` is the
+// state that is added to; null means `state` itself (in place).  On the tensor-core path everything
+// runs in one launch.
 int run_passes(const Problem& p, const void* k, const void* v, const void* q, void* o, float* state, bool accumulate,
-               float eps, void* workspace, cudaStream_t stream) {
+               float eps, void* workspace, cudaStream_t stream, const float* base = nullptr) {
   if (umma_supported(p)) {
-    UmmaCall c{k, v, q, o, state, accumulate, eps};
+    UmmaCall c{k, v, q, o, state, base, accumulate, eps};
     return umma_run(p, c, workspace, stream);
+  }
+  if (k && accumulate && base && base != state) {
+    if (cudaMemcpyAsync(state, base, state_bytes_of(p), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+      return LINATTN_ERR_CUDA;
   }
   if (k) {
     int st = cuda_status(fma_state(p, k, v, state, accumulate, partials_of(workspace), stream));
@@ -350,6 +355,23 @@ int blocklin_step(blocklin_cache* cache, int64_t T_b, const void* q_blk, const v
   int st = resolve(&cache->desc, T_b, &p);
   if (st != LINATTN_OK) return st;
   return step_impl(cache, p, q_blk, k_blk, v_blk, o_blk, (cudaStream_t)stream);
+}
+
+int blocklin_peek(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
+                  void* o_blk, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  Problem p;
+  int st = resolve(&cache->desc, T_b, &p);
+  if (st != LINATTN_OK) return st;
+  if (p.N > 0 && (!q_blk || !k_blk || !v_blk || !o_blk)) return LINATTN_ERR_INVALID_ARG;
+  if (o_blk && (o_blk == q_blk || o_blk == k_blk || o_blk == v_blk)) return LINATTN_ERR_INVALID_ARG;
+  if ((st = check_alignment(p, q_blk, k_blk, v_blk, o_blk)) != LINATTN_OK) return st;
+  if (cache->workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  if (p.N == 0) return LINATTN_OK;
+  // cache + state(block) goes to the state slot of the workspace; the cache itself is only read
+  float* tmp = reinterpret_cast<float*>(static_cast<char*>(cache->workspace) + state_slot_offset(p));
+  return run_passes(p, k_blk, v_blk, q_blk, o_blk, tmp, true, cache->eps, cache->workspace, (cudaStream_t)stream,
+                    cache->state);
 }
 
 int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,

@@ -54,7 +54,8 @@ struct UmmaCall {
   const void* v;
   const void* q;
   void* o;
-  float* state;     // written by the state pass (on top of its contents when `accumulate`), read by the apply pass
+  float* state;     // written by the state pass, read by the apply pass
+  const float* state_base;  // `accumulate`: the reduce adds the new state to this one (may be `state` itself)
   bool accumulate;
   float eps;
 };

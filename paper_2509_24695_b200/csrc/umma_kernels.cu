@@ -169,8 +169,9 @@ struct FusedParams {
   int B, H, HG;            // HG: head groups per batch entry = ceil(H / G)
   Sched sa, sc;            // state pass (64-token stages) and apply pass (128-token tiles)
   int do_state, do_apply;
-  int accumulate;          // reduce on top of the existing state
-  float* state;            // [B][H][(d+1)][d]
+  int accumulate;          // reduce on top of state_base
+  float* state;            // [B][H][(d+1)][d]: written by the reduce, read by the apply pass
+  const float* state_base; // the state the new one is added to (the cache; may be `state` itself)
   float* partials;         // one record of G head-states per (CTA, unit) segment of the state pass
   float eps;
   WorkspaceCtrl* ctrl;
@@ -279,7 +280,7 @@ __device__ void reduce_slice(const FusedParams& p) {
     const int b = bh / p.H, h = bh % p.H;
     const int u = b * p.HG + h / C::G, g = h % C::G;
     const float4* src = reinterpret_cast<const float4*>(p.partials) + (size_t)g * E4 + e;
-    float4 sum = p.accumulate ? __ldcg(state4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 sum = p.accumulate ? __ldcg(reinterpret_cast<const float4*>(p.state_base) + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
     // every record of the unit, column CTAs first, then the trailing CTAs; the loads of a batch are
     // independent and issued together, the adds keep that fixed order
     int r_lo = 0, ntrail = 0;
@@ -828,6 +829,7 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   fp.sc = make_sched(U, (p.N + kTileApply - 1) / kTileApply, sms, 2);
   fp.do_state = do_state; fp.do_apply = do_apply; fp.accumulate = c.accumulate ? 1 : 0;
   fp.state = c.state;
+  fp.state_base = c.state_base ? c.state_base : c.state;
   fp.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + LINATTN_WORKSPACE_CTRL_BYTES);
   fp.eps = c.eps;
   fp.ctrl = static_cast<WorkspaceCtrl*>(workspace);

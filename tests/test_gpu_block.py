@@ -147,3 +147,31 @@ def test_block_errors(la):
         assert err.status == -4
     assert cache.step(x[:, :0], x[:, :0].clone(), x[:, :0].clone()).shape[1] == 0
     assert cache.info()["blocks_seen"] in (0, 1)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 112), ("bf16", 64), ("f32", 112), ("bf16", 40)])
+def test_denoise_loop_reads_without_committing(la, orc, dtype, d):
+    """Algorithm 1: every denoising step of a block reads the cache together with the (noisy) block itself
+    but leaves the cache as it was; only the clean block is committed, once."""
+    import torch
+
+    B, H, T_b, M, T = 1, 3, 300, 3, 3
+    check = assert_parity_bf16 if dtype == "bf16" else assert_parity_f32
+    cache = la.BlockLinCache(B, H, d, tdtype(dtype), "cuda", max_T_b=T_b, eps=EPS)
+    S, z = orc.new_cache(B, H, d)
+    for blk in range(M):
+        before = cache.state.clone()
+        for j in range(T):  # noisy versions of the block: other values each time
+            q, k, v = gen(B, T_b, H, d, 3400 + 10 * blk + j, dtype)
+            o = cache.peek(to_dev(q), to_dev(k), to_dev(v))
+            ref = orc.block_step((S.copy(), z.copy()), q, k, v, EPS)   # the oracle's step on a COPY of its cache
+            check(to_f64(o), ref, f"peek block {blk} step {j}")
+            assert torch.equal(cache.state, before), "a read-only step changed the cache"
+            assert cache.info()["blocks_seen"] == blk
+        q, k, v = gen(B, T_b, H, d, 3500 + blk, dtype)               # the clean block
+        o_peek = cache.peek(to_dev(q), to_dev(k), to_dev(v))
+        o_step = cache.step(to_dev(q), to_dev(k), to_dev(v))
+        assert torch.equal(o_peek, o_step)                            # same arithmetic, committed or not
+        orc.block_step((S, z), q, k, v, EPS, want_o=False)
+        assert_state_close(to_f64(cache.state), S, z, 1e-5, f"cache after block {blk}")
+    assert cache.info()["blocks_seen"] == M
