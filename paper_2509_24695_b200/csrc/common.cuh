@@ -47,7 +47,7 @@ cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* sta
                       float* partials, cudaStream_t stream);
 cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream);
 
-// ---- tensor-core (tcgen05 + TMA) kernel, bf16, d in {64, 112, 128} ----
+// ---- tensor-core (tcgen05 + TMA) kernel, bf16, d in {32 (heads contiguous), 64, 112, 128} ----
 // One launch runs the state pass (k, v non-null), the apply pass (q, o non-null), or both back to back.
 struct UmmaCall {
   const void* k;

@@ -22,8 +22,8 @@
 // The first Q tiles of the apply pass are fetched before the grid barriers (Q does not depend on the
 // state), so HBM stays busy while the partials are reduced.
 //
-// Head dim 64 packs two heads into one 128-feature operand (the cross-head blocks of the product are
-// ignored / zero); 112 pads to 128 through TMA out-of-bounds zero fill.
+// Head dims 32 and 64 pack four / two heads into one 128-feature operand (the cross-head blocks of the
+// product are ignored / zero); 112 pads to 128 through TMA out-of-bounds zero fill.
 //
 // Warp roles (352 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 ReLU
 // pass, warps 6-9 epilogue, warp 10 output stores.  All cross-role synchronisation is by mbarriers
@@ -53,7 +53,7 @@ constexpr int kAccStride = 256;     // TMEM columns between the two accumulator 
 
 template <int D>
 struct Cfg {
-  static constexpr int G = D == 64 ? 2 : 1;                  // heads packed into one 128-feature operand
+  static constexpr int G = D == 32 ? 4 : D == 64 ? 2 : 1;   // heads packed into one 128-feature operand
   static constexpr int FEAT = G * D;                         // 112 or 128 live features per group
   static constexpr int KSTEPS = FEAT / 16;                   // apply: K steps over features
   static constexpr int ZROW = D == 112 ? 112 : 128;          // apply: accumulator column of the first denominator
@@ -181,7 +181,8 @@ struct FusedParams {
 template <int D>
 __device__ __forceinline__ void box_coords(int box, int hg, int& c0, int& c1) {
   if (Cfg<D>::G == 1) { c0 = 64 * box; c1 = hg; }
-  else { c0 = 0; c1 = 2 * hg + box; }
+  else if (Cfg<D>::G == 2) { c0 = 0; c1 = 2 * hg + box; }
+  else { c0 = 128 * hg + 64 * box; c1 = 0; }  // d = 32: the map sees a token's heads as one row of H*32 features
 }
 
 __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
@@ -792,6 +793,12 @@ bool make_map(CUtensorMap* map, const Problem& p, const void* base, int box_d, i
   if (!fn) return false;
   cuuint64_t dims[4] = {(cuuint64_t)p.d, (cuuint64_t)p.H, (cuuint64_t)p.N, (cuuint64_t)p.B};
   cuuint64_t strides[3] = {(cuuint64_t)p.sh * 2, (cuuint64_t)p.sn * 2, (cuuint64_t)p.sb * 2};
+  if (p.d == 32) {
+    // A 64-byte box row would be padded to the 128-byte swizzle pitch, so with d = 32 (heads contiguous:
+    // stride_h = 32) the heads of a token are one row of H*32 features and a box takes 64 of them (two heads).
+    dims[0] = (cuuint64_t)p.H * 32; dims[1] = 1;
+    strides[0] = (cuuint64_t)p.sn * 2;
+  }
   cuuint32_t box[4] = {(cuuint32_t)box_d, (cuuint32_t)box_h, (cuuint32_t)box_tokens, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
@@ -814,7 +821,7 @@ int sm_count() {
   return cached[dev];
 }
 
-inline int groups_of(int d) { return d == 64 ? 2 : 1; }
+inline int groups_of(int d) { return d == 32 ? 4 : d == 64 ? 2 : 1; }
 
 template <int D>
 int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
@@ -866,9 +873,8 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
 }  // namespace
 
 bool umma_supported(const Problem& p) {
-  // d = 32 is not taken yet: a 64-byte inner TMA box is padded to the 128-byte swizzle pitch in shared
-  // memory, so four heads cannot be packed into one operand row with this layout.
-  return p.dtype == LINATTN_BF16 && (p.d == 64 || p.d == 112 || p.d == 128) &&
+  // d = 32 packs four heads into one operand row, which needs the heads of a token to be contiguous
+  return p.dtype == LINATTN_BF16 && (p.d == 64 || p.d == 112 || p.d == 128 || (p.d == 32 && p.sh == 32)) &&
          p.N < (1ll << 31) && p.sh * 2 < (1ll << 40) && p.sn * 2 < (1ll << 40) && p.sb * 2 < (1ll << 40);
 }
 
@@ -882,6 +888,7 @@ size_t umma_partial_bytes(const Problem& p) {
 int umma_run(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
   if (p.N == 0 || (!c.k && !c.q)) return LINATTN_OK;
   switch (p.d) {
+    case 32: return launch_fused<32>(p, c, workspace, stream);
     case 64: return launch_fused<64>(p, c, workspace, stream);
     case 112: return launch_fused<112>(p, c, workspace, stream);
     case 128: return launch_fused<128>(p, c, workspace, stream);
