@@ -155,7 +155,9 @@ LINATTN_API int linattn_apply(const linattn_desc* desc, int64_t N, const void* q
  * `dev_staging` (DEVICE, 256-byte aligned) must hold linattn_forward_host_bytes() bytes: four dense
  * [B,N,H,d] tensors plus the forward's workspace; its control block must have been zeroed once with
  * linattn_workspace_init(dev_staging, ...).  Host tensors are dense [B,N,H,d] (the descriptor's
- * strides must be 0).  The host buffers may be reused once `stream` has been synchronised. */
+ * strides must be 0).  Q is uploaded and O downloaded in token chunks, the downloads on a second stream
+ * that the library keeps per device, so that the two copy directions overlap; `stream` is made to wait
+ * for the last download, so the host buffers may be reused once `stream` has been synchronised. */
 LINATTN_API int linattn_forward_host_bytes(const linattn_desc* desc, int64_t N, size_t* bytes);
 LINATTN_API int linattn_forward_host(const linattn_desc* desc, int64_t N, const void* q_host, const void* k_host,
                                      const void* v_host, void* o_host, float eps, void* dev_staging,

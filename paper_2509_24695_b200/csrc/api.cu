@@ -111,6 +111,30 @@ static void* static_scratch_address() {
   return cached[dev];
 }
 
+// Host-side plumbing of linattn_forward_host: a second stream for the downloads and the events that
+// order it against the caller's stream (no device memory), created once per device.
+constexpr int kHostChunks = 8;
+struct HostPipe {
+  cudaStream_t down;
+  cudaEvent_t chunk_done[kHostChunks + 1];
+  cudaEvent_t all_down;
+};
+static HostPipe* host_pipe() {
+  static HostPipe pipes[64];
+  static bool ready[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!ready[dev]) {
+    HostPipe& hp = pipes[dev];
+    if (cudaStreamCreateWithFlags(&hp.down, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    for (cudaEvent_t& ev : hp.chunk_done)
+      if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&hp.all_down, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    ready[dev] = true;
+  }
+  return &pipes[dev];
+}
+
 struct blocklin_cache {
   uint32_t magic;
   linattn_desc desc;
@@ -287,14 +311,43 @@ int linattn_forward_host(const linattn_desc* desc, int64_t N, const void* q_host
   void* dv = base + ws + 2 * tensor;
   void* dout = base + ws + 3 * tensor;
   cudaStream_t s = (cudaStream_t)stream;
-  // K and V first: the state pass needs them; Q is only needed by the apply pass
+  // K and V first: the state pass needs them.  Then Q goes up and O comes down in token chunks, the
+  // download of chunk c (on a second stream) running under the upload and the apply pass of chunk c+1:
+  // the two copy directions do not share an engine.
+  HostPipe* pipe = host_pipe();
+  if (!pipe) return LINATTN_ERR_CUDA;
   cudaError_t e = cudaMemcpyAsync(dk, k_host, bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, bytes, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, bytes, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return LINATTN_ERR_CUDA;
-  st = linattn_forward(desc, N, dq, dk, dv, dout, eps, dev_staging, ws, stream);
+  float* state = reinterpret_cast<float*>(base + state_slot_offset(p));
+  st = run_passes(p, dk, dv, nullptr, nullptr, state, false, 0.f, dev_staging, s);
   if (st != LINATTN_OK) return st;
-  return cuda_status(cudaMemcpyAsync(o_host, dout, bytes, cudaMemcpyDeviceToHost, s));
+  const long long chunk_tokens = N >= 8 * 1024 ? (((N + kHostChunks - 1) / kHostChunks + 127) / 128) * 128 : N;
+  const size_t row = (size_t)p.H * p.d * esz;  // bytes of one token
+  int c = 0;
+  for (long long n0 = 0; n0 < N; n0 += chunk_tokens, ++c) {
+    const long long nc = N - n0 < chunk_tokens ? N - n0 : chunk_tokens;
+    const size_t off = (size_t)n0 * row;
+    // dense [B, N, H, d]: the chunk is B pieces of nc*row bytes, N*row bytes apart
+    e = cudaMemcpy2DAsync(static_cast<char*>(dq) + off, (size_t)N * row, static_cast<const char*>(q_host) + off,
+                          (size_t)N * row, (size_t)nc * row, p.B, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return LINATTN_ERR_CUDA;
+    Problem pc = p;
+    pc.N = nc;  // strides stay those of the whole tensor
+    st = run_passes(pc, nullptr, nullptr, static_cast<char*>(dq) + off, static_cast<char*>(dout) + off, state, false, eps,
+                    dev_staging, s);
+    if (st != LINATTN_OK) return st;
+    if (cudaEventRecord(pipe->chunk_done[c], s) != cudaSuccess ||
+        cudaStreamWaitEvent(pipe->down, pipe->chunk_done[c], 0) != cudaSuccess)
+      return LINATTN_ERR_CUDA;
+    e = cudaMemcpy2DAsync(static_cast<char*>(o_host) + off, (size_t)N * row, static_cast<char*>(dout) + off,
+                          (size_t)N * row, (size_t)nc * row, p.B, cudaMemcpyDeviceToHost, pipe->down);
+    if (e != cudaSuccess) return LINATTN_ERR_CUDA;
+  }
+  // the caller's stream is complete only when the last download is
+  if (cudaEventRecord(pipe->all_down, pipe->down) != cudaSuccess || cudaStreamWaitEvent(s, pipe->all_down, 0) != cudaSuccess)
+    return LINATTN_ERR_CUDA;
+  return LINATTN_OK;
 }
 
 int blocklin_cache_bytes(const linattn_desc* desc, int64_t max_T_b, size_t* state_bytes, size_t* workspace_bytes) {

@@ -190,3 +190,24 @@ def test_zero_tokens_and_errors(la):
         la.linattn_forward(x, x.clone(), x.clone(), EPS, workspace=ws)
     assert e.value.status == -4
     assert la.workspace_status(la.new_workspace(x)) == 0
+
+
+@pytest.mark.parametrize("shape", [(1, 9000, 3, 112), (2, 8300, 2, 64), (1, 500, 2, 112)],
+                         ids=lambda s: "B%d_N%d_H%d_d%d" % s)
+def test_forward_from_host_buffers(la, orc, shape):
+    """The host-buffer entry point (chunked upload of Q / download of O) gives the device path's bits."""
+    import torch
+
+    B, N, H, d = shape
+    q, k, v = gen(B, N, H, d, 2300 + N, "bf16")
+    pin = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    qp, kp, vp = pin(q), pin(k), pin(v)
+    op = torch.zeros_like(qp).pin_memory()
+    hf = la.HostForward(B, N, H, d, torch.bfloat16, "cuda")
+    for _ in range(2):  # twice: the staging area and the second stream are reused
+        op.zero_()
+        hf(qp, kp, vp, op, EPS)
+        torch.cuda.synchronize()
+        ref_dev = la.linattn_forward(to_dev(q), to_dev(k), to_dev(v), EPS)
+        assert torch.equal(op.cuda(), ref_dev)
+    assert_parity_bf16(to_f64(op), orc.forward(q, k, v, EPS), f"host forward {shape}")
