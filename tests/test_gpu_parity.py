@@ -211,3 +211,22 @@ def test_forward_from_host_buffers(la, orc, shape):
         ref_dev = la.linattn_forward(to_dev(q), to_dev(k), to_dev(v), EPS)
         assert torch.equal(op.cuda(), ref_dev)
     assert_parity_bf16(to_f64(op), orc.forward(q, k, v, EPS), f"host forward {shape}")
+
+
+def test_bounded_wait_reports_timeout_and_the_context_survives(la):
+    """Every device-side wait is bounded.  A grid-barrier word that can never reach its target (the
+    workspace's control block is required to start at zero; here it does not) makes the wait run out after
+    about a second: the kernel returns, LINATTN_ERR_TIMEOUT is in the status word, nothing traps, and
+    after re-initialising the workspace the same call works."""
+    import torch
+
+    q, k, v = (to_dev(x) for x in gen(1, 2000, 2, 112, 97, "bf16"))
+    ws = la.new_workspace(q)
+    good = la.linattn_state(k, v, workspace=ws).clone()
+    ctrl = ws[:4096].view(torch.int32)
+    ctrl[16] = 0x4000           # arrival count of the barrier word: never equals grid - 1 again
+    la.linattn_state(k, v, workspace=ws)
+    assert la.workspace_status(ws) == -6
+    la.load_library().linattn_workspace_init(ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
+    assert la.workspace_status(ws) == 0
+    assert torch.equal(la.linattn_state(k, v, workspace=ws), good)
