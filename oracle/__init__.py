@@ -51,6 +51,8 @@ def _bind(path: str):
     lib.oracle_quadratic.argtypes = [sp, vp, vp, vp, f64, i64, dp]
     lib.oracle_block_step.argtypes = [sp, vp, vp, vp, f64, dp, dp, dp]
     lib.oracle_block_masked.argtypes = [sp, vp, vp, vp, f64, i64, dp]
+    lib.oracle_rope_forward.argtypes = [sp, vp, vp, vp, dp, dp, f64, dp]
+    lib.oracle_rope_quadratic.argtypes = [sp, vp, vp, vp, dp, dp, f64, dp]
     lib.oracle_cache_bytes.argtypes = [i64, i64, i64]
     lib.oracle_cache_bytes.restype = i64
     return lib
@@ -112,6 +114,18 @@ class Oracle:
         s = self._shape(q, k, v)
         o = np.empty((s.B, s.N, s.H, s.d))
         self._lib.oracle_block_masked(ctypes.byref(s), q.ctypes.data, k.ctypes.data, v.ctypes.data, eps, T_b, self._dp(o))
+        return o
+
+    def rope_forward(self, q, k, v, cos, sin, eps, quadratic: bool = False):
+        """Eq. 2 with rotary factors in the numerator only.  cos, sin: [N, d//2] (any float dtype; widened
+        exactly to fp64), the rotation of feature pair (2p, 2p+1) of token n."""
+        s = self._shape(q, k, v)
+        cs = np.ascontiguousarray(cos, dtype=np.float64)
+        sn = np.ascontiguousarray(sin, dtype=np.float64)
+        assert cs.shape == sn.shape == (s.N, s.d // 2)
+        o = np.empty((s.B, s.N, s.H, s.d))
+        fn = self._lib.oracle_rope_quadratic if quadratic else self._lib.oracle_rope_forward
+        fn(ctypes.byref(s), q.ctypes.data, k.ctypes.data, v.ctypes.data, self._dp(cs), self._dp(sn), eps, self._dp(o))
         return o
 
     def new_cache(self, B, H, d):

@@ -211,5 +211,91 @@ void oracle_block_masked(const oracle_shape* s, const void* q, const void* k, co
   }
 }
 
+/* ---- Eq. 2 with the rotary factors (its right-hand form) ----
+ *
+ *   o_n = RoPE_n(phi(q_n)) ( sum_m RoPE_m(phi(k_m))^T v_m ) / ( phi(q_n) . sum_m phi(k_m) + eps )
+ *
+ * The rotation is applied AFTER the ReLU and only in the numerator; the denominator uses the plain
+ * features, so it stays non-negative (Sec. 3.1).  RoPE_n rotates the feature pair (2p, 2p+1) of token n by
+ * an angle given through its cosine and sine: (a, b) -> (a c - b s, a s + b c), c = cs[n][p], s = sn[n][p]
+ * (tables [N][d/2], shared by all batch entries and heads).  How the angles depend on the token's
+ * (t, h, w) position is the caller's business: the paper does not give its 3D split or base frequency. */
+static void rope_features(const oracle_shape* s, const void* x, int64_t base, const double* cs, const double* sn,
+                          int64_t n, double* plain, double* rot) {
+  const int64_t d = s->d, half = d / 2;
+  for (int64_t i = 0; i < d; ++i) plain[i] = relu(load_elem(x, s->dtype, base + i));
+  for (int64_t p = 0; p < half; ++p) {
+    const double c = cs[n * half + p], t = sn[n * half + p];
+    rot[2 * p] = plain[2 * p] * c - plain[2 * p + 1] * t;
+    rot[2 * p + 1] = plain[2 * p] * t + plain[2 * p + 1] * c;
+  }
+  if (d & 1) rot[d - 1] = plain[d - 1]; /* an unpaired last feature is not rotated */
+}
+
+/* Linear form: S from the rotated keys, z from the plain keys; numerator from the rotated query, denominator
+ * from the plain query.  o: [B,N,H,d] dense fp64. */
+void oracle_rope_forward(const oracle_shape* s, const void* q, const void* k, const void* v, const double* cs,
+                         const double* sn, double eps, double* o) {
+  const int64_t d = s->d, BH = s->B * s->H;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t u = 0; u < BH; ++u) {
+    const int64_t b = u / s->H, h = u % s->H;
+    double* S = (double*)calloc((size_t)(d * d + 3 * d), sizeof(double));
+    double* z = S + d * d;
+    double* plain = z + d;
+    double* rot = plain + d;
+    for (int64_t n = 0; n < s->N; ++n) {
+      const int64_t base = at(s, b, n, h);
+      rope_features(s, k, base, cs, sn, n, plain, rot);
+      for (int64_t i = 0; i < d; ++i) {
+        z[i] += plain[i];
+        for (int64_t j = 0; j < d; ++j) S[i * d + j] += rot[i] * load_elem(v, s->dtype, base + j);
+      }
+    }
+    for (int64_t n = 0; n < s->N; ++n) {
+      double* o_row = o + ((b * s->N + n) * s->H + h) * d;
+      rope_features(s, q, at(s, b, n, h), cs, sn, n, plain, rot);
+      double den = 0.0;
+      for (int64_t j = 0; j < d; ++j) o_row[j] = 0.0;
+      for (int64_t i = 0; i < d; ++i) {
+        den += plain[i] * z[i];
+        for (int64_t j = 0; j < d; ++j) o_row[j] += rot[i] * S[i * d + j];
+      }
+      den += eps;
+      for (int64_t j = 0; j < d; ++j) o_row[j] /= den;
+    }
+    free(S);
+  }
+}
+
+/* Quadratic form of the same: w_num[n][m] = RoPE_n(phi(q_n)) . RoPE_m(phi(k_m)), w_den[n][m] = phi(q_n) . phi(k_m),
+ * o_n = sum_m w_num[n][m] v_m / (sum_m w_den[n][m] + eps).  O(N^2 d): tiny inputs only. */
+void oracle_rope_quadratic(const oracle_shape* s, const void* q, const void* k, const void* v, const double* cs,
+                           const double* sn, double eps, double* o) {
+  const int64_t d = s->d, BH = s->B * s->H;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t u = 0; u < BH; ++u) {
+    const int64_t b = u / s->H, h = u % s->H;
+    double* buf = (double*)calloc((size_t)(4 * d), sizeof(double));
+    double *qp = buf, *qr = buf + d, *kp = buf + 2 * d, *kr = buf + 3 * d;
+    for (int64_t n = 0; n < s->N; ++n) {
+      double* o_row = o + ((b * s->N + n) * s->H + h) * d;
+      rope_features(s, q, at(s, b, n, h), cs, sn, n, qp, qr);
+      double wden = 0.0;
+      for (int64_t j = 0; j < d; ++j) o_row[j] = 0.0;
+      for (int64_t m = 0; m < s->N; ++m) {
+        const int64_t kb = at(s, b, m, h);
+        rope_features(s, k, kb, cs, sn, m, kp, kr);
+        double wn = 0.0;
+        for (int64_t i = 0; i < d; ++i) { wn += qr[i] * kr[i]; wden += qp[i] * kp[i]; }
+        for (int64_t j = 0; j < d; ++j) o_row[j] += wn * load_elem(v, s->dtype, kb + j);
+      }
+      wden += eps;
+      for (int64_t j = 0; j < d; ++j) o_row[j] /= wden;
+    }
+    free(buf);
+  }
+}
+
 /* Bytes of the fp64 cache this oracle keeps for a stream: depends on (B,H,d) only (Table 1). */
 int64_t oracle_cache_bytes(int64_t B, int64_t H, int64_t d) { return B * H * (d * d + d) * (int64_t)sizeof(double); }

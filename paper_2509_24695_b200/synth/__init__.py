@@ -161,3 +161,24 @@ def qkv_block(w: Workload, blk: int, dtype: str = "bf16", n_tokens: int | None =
             gauss((T, w.H, w.d), w.seed, t, scale=w.scale, start=(b * w.N + blk * w.T_b) * C, dtype=dtype, out=a[b])
         outs.append(a)
     return tuple(outs)
+
+
+def rope_table(T: int, Hh: int, Ww: int, d: int, base: float = 10000.0):
+    """cos, sin tables ``[T*Hh*Ww, d//2]`` (float32) of a 3D rotary embedding for tokens ordered (t, h, w).
+
+    The paper gives neither the split of the head dim over the three axes nor the base frequency, so this
+    is only a plausible input for tests and measurements: of the d//2 feature pairs, d//6 go to the height
+    and to the width axis each and the rest to time; pair i of an axis with n_a pairs turns by
+    ``pos * base**(-i / n_a)`` (the rotary formula of Su et al., per axis).
+    """
+    half = d // 2
+    n_hw = d // 6
+    n_t = half - 2 * n_hw
+    t, h, w = np.meshgrid(np.arange(T), np.arange(Hh), np.arange(Ww), indexing="ij")
+    cols = []
+    for pos, n_a in ((t, n_t), (h, n_hw), (w, n_hw)):
+        freq = base ** (-np.arange(n_a, dtype=np.float64) / max(n_a, 1))
+        cols.append(pos.reshape(-1, 1).astype(np.float64) * freq[None, :])
+    theta = np.concatenate(cols, axis=1)
+    assert theta.shape == (T * Hh * Ww, half)
+    return np.cos(theta).astype(np.float32), np.sin(theta).astype(np.float32)

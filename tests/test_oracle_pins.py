@@ -257,9 +257,86 @@ def pin_strides_and_rows(o):
     assert np.array_equal(S1[0, 0], want) and np.array_equal(z1[0, 0], [2.0, 0.0, 0.0])
 
 
+def _angles(N, half, seed, scale=3.0):
+    th = synth.gauss((N, half), seed, 7, dtype="f32").astype(np.float64) * scale
+    return np.cos(th), np.sin(th), th
+
+
+def pin_rope_closed_form_d2(o):
+    """d = 2, phi(q) = phi(k) = (1, 0): the rotated dot product is cos(theta_n - theta_m), the plain one is 1,
+    so o_n = sum_m cos(theta_n - theta_m) v_m / (N + eps)  (Eq. 2, right-hand form)."""
+    N = 5
+    th = np.array([0.0, 0.3, -1.1, 2.0, np.pi / 2])
+    q = np.zeros((1, N, 1, 2)); q[..., 0] = 1.0; q[..., 1] = -2.0      # the negative entry is cut by the ReLU
+    k = q.copy()
+    v = _rand((1, N, 1, 2), 81, 3)
+    want = (np.cos(th[:, None] - th[None, :]) @ v[0, :, 0]) / (N + 0.25)
+    for quad in (False, True):
+        out = o.rope_forward(q, k, v, np.cos(th)[:, None], np.sin(th)[:, None], 0.25, quadratic=quad)
+        assert np.allclose(out[0, :, 0], want, rtol=0, atol=1e-14)
+    # table column p belongs to feature pair (2p, 2p+1): with d = 4 and only features 0, 1 alive, angles in
+    # column 0 act as above and angles in column 1 do nothing
+    q4 = np.zeros((1, N, 1, 4)); q4[..., 0] = 1.0
+    v4 = _rand((1, N, 1, 4), 82, 3)
+    zero = np.zeros(N)
+    out = o.rope_forward(q4, q4.copy(), v4, np.stack([np.cos(th), np.cos(zero)], 1), np.stack([np.sin(th), np.sin(zero)], 1), 0.25)
+    assert np.allclose(out[0, :, 0], (np.cos(th[:, None] - th[None, :]) @ v4[0, :, 0]) / (N + 0.25), rtol=0, atol=1e-14)
+    out = o.rope_forward(q4, q4.copy(), v4, np.stack([np.cos(zero), np.cos(th)], 1), np.stack([np.sin(zero), np.sin(th)], 1), 0.25)
+    assert np.allclose(out[0, :, 0], np.broadcast_to(v4[0, :, 0].sum(0) / (N + 0.25), (N, 4)), rtol=0, atol=1e-14)
+    # a quarter turn on the key only: (1,0) -> (0,1), orthogonal to the unrotated query: numerator 0, denominator not
+    th2 = np.array([0.0, np.pi / 2])
+    out = o.rope_forward(q[:, :2].copy(), k[:, :2].copy(), np.ones((1, 2, 1, 2)), np.cos(th2)[:, None], np.sin(th2)[:, None], 0.0)
+    assert np.allclose(out[0, 0, 0], [0.5, 0.5], atol=1e-14) and np.allclose(out[0, 1, 0], [0.5, 0.5], atol=1e-14)
+    # rotation direction: (a, b) -> (a c - b s, a s + b c).  k = (0, 1) turned by +90 deg becomes (-1, 0)
+    qd = np.array([1.0, 0.0]).reshape(1, 1, 1, 2); kd = np.array([0.0, 1.0]).reshape(1, 1, 1, 2)
+    q2 = np.concatenate([qd, qd], 1); k2 = np.concatenate([kd, kd], 1); v2 = np.array([[1.0, 0.0], [0.0, 1.0]]).reshape(1, 2, 1, 2)
+    out = o.rope_forward(q2, k2, v2, np.array([[1.0], [0.0]]), np.array([[0.0], [1.0]]), 1.0)
+    # token 0 (angle 0): rotated q = (1,0); rotated keys: (0,1) and (-1,0): weights 0 and -1; plain weights 0, 0
+    assert np.allclose(out[0, 0, 0], [0.0, -1.0], atol=1e-14)
+
+
+def pin_rope_reduces_to_plain(o):
+    """Zero angles, or one common angle per feature pair for all tokens (relative angle zero), give Eq. 2
+    without rotary factors: the numerator only sees angle differences and the denominator sees none."""
+    B, N, H, d = 2, 9, 2, 6
+    q, k, v = _qkv(B, N, H, d, 83)
+    plain = o.forward(q, k, v, EPS)
+    one, zero = np.ones((N, d // 2)), np.zeros((N, d // 2))
+    assert np.array_equal(o.rope_forward(q, k, v, one, zero, EPS), plain)
+    delta = np.array([0.7, -2.0, 1.3])
+    cs, sn = np.broadcast_to(np.cos(delta), (N, 3)), np.broadcast_to(np.sin(delta), (N, 3))
+    assert np.allclose(o.rope_forward(q, k, v, cs, sn, EPS), plain, rtol=1e-12, atol=1e-13)
+    # ... and with real angles the result differs from the plain one
+    cs, sn, _ = _angles(N, 3, 84)
+    assert np.abs(o.rope_forward(q, k, v, cs, sn, EPS) - plain).max() > 1e-3
+
+
+def pin_rope_linear_equals_quadratic_and_shift(o):
+    for (B, N, H, d, seed) in [(1, 1, 1, 2, 85), (2, 7, 3, 4, 86), (1, 33, 2, 14, 87), (1, 12, 1, 5, 88)]:
+        q, k, v = _qkv(B, N, H, d, seed)
+        cs, sn, th = _angles(N, d // 2, seed + 100)
+        lin = o.rope_forward(q, k, v, cs, sn, EPS)
+        quad = o.rope_forward(q, k, v, cs, sn, EPS, quadratic=True)
+        assert np.allclose(lin, quad, rtol=1e-11, atol=1e-12)
+        # only angle differences matter: a common offset per pair changes nothing
+        off = np.linspace(-1.0, 2.0, d // 2)
+        assert np.allclose(o.rope_forward(q, k, v, np.cos(th + off), np.sin(th + off), EPS), lin, rtol=1e-11, atol=1e-12)
+        # the denominator is the plain one: scaling V scales the output, and sum_m w_den is that of the plain form
+        ones = np.ones_like(v)
+        den_ratio = o.rope_forward(q, k, ones, cs, sn, EPS)          # = sum_m w_num / (sum_m w_den + eps), same in every column
+        assert np.allclose(den_ratio, den_ratio[..., :1], rtol=1e-12, atol=1e-13)
+    # each head and batch entry is independent, the table is shared
+    q, k, v = _qkv(2, 6, 2, 4, 89)
+    cs, sn, _ = _angles(6, 2, 90)
+    full = o.rope_forward(q, k, v, cs, sn, EPS)
+    part = o.rope_forward(q[1:, :, 1:].copy(), k[1:, :, 1:].copy(), v[1:, :, 1:].copy(), cs, sn, EPS)
+    assert np.array_equal(full[1:, :, 1:], part)
+
+
 PINS = [pin_hand_worked_example, pin_exact_rational, pin_linear_equals_quadratic, pin_bf16_decode_and_tiny_config,
         pin_constant_v, pin_single_token, pin_one_hot_is_segment_mean, pin_invariances, pin_sign, pin_convexity,
-        pin_block_forms_agree, pin_cache_size_constant, pin_strides_and_rows]
+        pin_block_forms_agree, pin_cache_size_constant, pin_strides_and_rows, pin_rope_closed_form_d2,
+        pin_rope_reduces_to_plain, pin_rope_linear_equals_quadratic_and_shift]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -302,6 +379,13 @@ MUTANTS = {
     "v_index_uses_i": ("Srow[j] += kp * load_elem(v, s->dtype, base + j);", "Srow[j] += kp * load_elem(v, s->dtype, base + i);"),
     "cache_bytes_grow": ("return B * H * (d * d + d) * (int64_t)sizeof(double);", "return B * H * (d * d) * (int64_t)sizeof(double);"),
     "state_not_zeroed": ("    memset(Su, 0, sizeof(double) * d * d);\n", ""),
+    "rope_before_relu_sign": ("rot[2 * p] = plain[2 * p] * c - plain[2 * p + 1] * t;", "rot[2 * p] = plain[2 * p] * c + plain[2 * p + 1] * t;"),
+    "rope_pairs_half_split": ("const double c = cs[n * half + p], t = sn[n * half + p];", "const double c = cs[n * half + (p + 1) % half], t = sn[n * half + (p + 1) % half];"),
+    "rope_in_denominator_linear": ("        z[i] += plain[i];\n", "        z[i] += rot[i];\n"),
+    "rope_den_uses_rotated_query": ("        den += plain[i] * z[i];\n", "        den += rot[i] * z[i];\n"),
+    "rope_state_from_plain_keys": ("S[i * d + j] += rot[i] * load_elem(v, s->dtype, base + j);", "S[i * d + j] += plain[i] * load_elem(v, s->dtype, base + j);"),
+    "rope_quadratic_den_rotated": ("wden += qp[i] * kp[i];", "wden += qr[i] * kr[i];"),
+    "rope_token_index": ("rope_features(s, k, base, cs, sn, n, plain, rot);", "rope_features(s, k, base, cs, sn, 0, plain, rot);"),
 }
 
 
