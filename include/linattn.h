@@ -114,6 +114,20 @@ LINATTN_API int linattn_workspace_status(const void* workspace, void* stream, in
 LINATTN_API int linattn_forward(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v, void* o,
                     float eps, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Eq. 2 as printed, with its rotary factors (Sec. 3.1): the rotation is applied after the ReLU and in the
+ * numerator only,
+ *     o_n = RoPE_n(phi(q_n)) ( sum_m RoPE_m(phi(k_m))^T v_m ) / ( phi(q_n) . sum_m phi(k_m) + eps ),
+ * so the denominator stays non-negative.  RoPE_n turns the feature pair (2p, 2p+1) of token n by the angle
+ * whose cosine and sine are rope_cos[n*(d/2) + p] and rope_sin[n*(d/2) + p]:
+ * (a, b) -> (a c - b s, a s + b c).  The tables are DEVICE fp32 arrays [N][d/2], 16-byte aligned, shared by
+ * all batch entries and heads; how the angles follow from a token's (t, h, w) position (the paper's 3D RoPE)
+ * is the caller's choice.  d must be even.  The workspace must hold linattn_rope_workspace_bytes() bytes
+ * (control block zeroed once with linattn_workspace_init). */
+LINATTN_API int linattn_rope_workspace_bytes(const linattn_desc* desc, int64_t N, size_t* bytes);
+LINATTN_API int linattn_forward_rope(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v,
+                                     void* o, float eps, const float* rope_cos, const float* rope_sin, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
 /* The state of Eq. 2 / Eq. 3 alone: state = (sum_n phi(k_n)^T v_n, sum_n phi(k_n)) in the layout above.
  * Deterministic: split-N partials are summed in a fixed order, so repeated calls give identical bits. */
 LINATTN_API int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void* v, float* state,

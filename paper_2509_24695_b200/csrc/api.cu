@@ -89,6 +89,23 @@ int run_passes(const Problem& p, const void* k, const void* v, const void* q, vo
   return LINATTN_OK;
 }
 
+// Workspace of the rotary entry point: [control block][split-N partials][one state].
+size_t rope_partial_bytes(const Problem& p) {
+  return sizeof(float) * (size_t)p.state_elems() * p.units() * fma_chunks(p.N);
+}
+size_t rope_state_offset(const Problem& p) { return round256(LINATTN_WORKSPACE_CTRL_BYTES + rope_partial_bytes(p)); }
+size_t rope_workspace_need(const Problem& p) { return round256(rope_state_offset(p) + state_bytes_of(p)); }
+
+// Eq. 2 with its rotary factors: state from the rotated keys (z from the plain ones), apply with the rotated
+// queries (denominator from the plain ones).
+int run_rope(const Problem& p, const void* q, const void* k, const void* v, void* o, float* state, float eps,
+             const float* rope_cos, const float* rope_sin, void* workspace, cudaStream_t stream) {
+  // the split-N scratch must hold the FMA path's partials too (workspace_need covers the larger of the two)
+  int st = cuda_status(fma_state(p, k, v, state, false, partials_of(workspace), stream, rope_cos, rope_sin));
+  if (st != LINATTN_OK) return st;
+  return cuda_status(fma_apply(p, q, state, o, eps, stream, rope_cos, rope_sin));
+}
+
 }  // namespace
 
 // Scratch of linattn_state_static_scratch: part of the library image, so no call has to allocate it.
@@ -273,6 +290,33 @@ int linattn_forward(const linattn_desc* desc, int64_t N, const void* q, const vo
   // the forward keeps its reduced state in the workspace, after the partials
   float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + state_slot_offset(p));
   return run_passes(p, k, v, q, o, state, false, eps, workspace, (cudaStream_t)stream);
+}
+
+int linattn_rope_workspace_bytes(const linattn_desc* desc, int64_t N, size_t* bytes) {
+  Problem p;
+  if (!bytes) return LINATTN_ERR_INVALID_ARG;
+  int st = resolve(desc, N, &p);
+  if (st != LINATTN_OK) return st;
+  *bytes = rope_workspace_need(p);
+  return LINATTN_OK;
+}
+
+int linattn_forward_rope(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v, void* o,
+                         float eps, const float* rope_cos, const float* rope_sin, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+  Problem p;
+  int st = resolve(desc, N, &p);
+  if (st != LINATTN_OK) return st;
+  if (!workspace) return LINATTN_ERR_INVALID_ARG;
+  if (p.d & 1) return LINATTN_ERR_UNSUPPORTED;  // the rotation pairs features (2p, 2p+1)
+  if (N > 0 && (!q || !k || !v || !o || !rope_cos || !rope_sin || o == q || o == k || o == v))
+    return LINATTN_ERR_INVALID_ARG;
+  if ((st = check_alignment(p, q, k, v, o)) != LINATTN_OK) return st;
+  if (!aligned16(workspace) || !aligned16(rope_cos) || !aligned16(rope_sin)) return LINATTN_ERR_BAD_ALIGNMENT;
+  if (workspace_bytes < rope_workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  if (N == 0) return LINATTN_OK;
+  float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + rope_state_offset(p));
+  return run_rope(p, q, k, v, o, state, eps, rope_cos, rope_sin, workspace, (cudaStream_t)stream);
 }
 
 uint64_t linattn_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }

@@ -43,9 +43,12 @@ inline int fma_chunks(long long N) {
 
 // ---- FMA kernels (fp32 I/O path, and bf16 shapes the tensor-core kernels do not take) ----
 // state_out = (accumulate ? state_out : 0) + state of tokens [0, N); partials is scratch.
+// rope_cos / rope_sin (both or neither): Eq. 2 with its rotary factors, tables [N][d/2] of the pair rotations.
 cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate,
-                      float* partials, cudaStream_t stream);
-cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream);
+                      float* partials, cudaStream_t stream, const float* rope_cos = nullptr,
+                      const float* rope_sin = nullptr);
+cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream,
+                      const float* rope_cos = nullptr, const float* rope_sin = nullptr);
 
 // ---- tensor-core (tcgen05 + TMA) kernel, bf16, d in {32 (heads contiguous), 64, 112, 128} ----
 // One launch runs the state pass (k, v non-null), the apply pass (q, o non-null), or both back to back.

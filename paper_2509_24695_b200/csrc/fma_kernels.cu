@@ -16,7 +16,6 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kPitch = 132;      // shared-memory row pitch in floats (128 + 4: breaks bank alignment of rows)
-constexpr int kStateTile = 32;   // tokens staged per iteration in the state kernel
 constexpr int kApplyTile = 64;   // tokens per CTA in the apply kernel
 
 template <typename T>
@@ -35,11 +34,16 @@ __device__ __forceinline__ void store_out<__nv_bfloat16>(__nv_bfloat16* p, float
 
 // grid (P, units).  R = ceil(d/16): each thread owns an R x R register tile of S:
 // rows i = ti + 16*r (key feature), columns j = tj + 16*c (value feature).
-template <typename T, int R>
+// ROPE (Eq. 2 with its rotary factors): S is built from the rotated phi(k) (pair (2p, 2p+1) of token n turned
+// by the angle whose cosine and sine are cs[n][p], sn[n][p]), z from the plain phi(k).
+template <typename T, int R, bool ROPE>
 __global__ void __launch_bounds__(kThreads)
-fma_state_partial(const T* __restrict__ k, const T* __restrict__ v, Problem p, int P, float* __restrict__ partials) {
+fma_state_partial(const T* __restrict__ k, const T* __restrict__ v, Problem p, int P, float* __restrict__ partials,
+                  const float* __restrict__ cs, const float* __restrict__ sn) {
+  constexpr int kStateTile = ROPE ? 16 : 32;  // tokens staged per iteration (three staging arrays with ROPE)
   __shared__ float Ks[kStateTile * kPitch];
   __shared__ float Vs[kStateTile * kPitch];
+  __shared__ float Zs[ROPE ? kStateTile * kPitch : 1];  // plain phi(k), for z
   const int d = p.d;
   const int u = blockIdx.y, c = blockIdx.x;
   const int b = u / p.H, h = u % p.H;
@@ -62,14 +66,21 @@ fma_state_partial(const T* __restrict__ k, const T* __restrict__ v, Problem p, i
     __syncthreads();
     for (int idx = tid; idx < kStateTile * 16 * R; idx += kThreads) {
       const int n = idx / (16 * R), e = idx % (16 * R);
-      float kv = 0.f, vv = 0.f;
+      float kv = 0.f, vv = 0.f, kplain = 0.f;
       if (n0 + n < n_end && e < d) {
         const long long off = base + (n0 + n) * p.sn + e;
-        kv = fmaxf(load_f32<T>(k + off), 0.f);  // phi = ReLU on the keys
+        kv = kplain = fmaxf(load_f32<T>(k + off), 0.f);  // phi = ReLU on the keys
         vv = load_f32<T>(v + off);
+        if (ROPE && (e ^ 1) < d) {  // rotate after the ReLU; an unpaired last feature stays
+          const float other = fmaxf(load_f32<T>(k + off + ((e ^ 1) - e)), 0.f);
+          const long long t = (n0 + n) * (long long)(d / 2) + e / 2;
+          const float c = cs[t], sgn = sn[t];
+          kv = (e & 1) ? other * sgn + kplain * c : kplain * c - other * sgn;
+        }
       }
       Ks[n * kPitch + e] = kv;
       Vs[n * kPitch + e] = vv;
+      if (ROPE) Zs[n * kPitch + e] = kplain;
     }
     __syncthreads();
 #pragma unroll 4
@@ -82,7 +93,7 @@ fma_state_partial(const T* __restrict__ k, const T* __restrict__ v, Problem p, i
       }
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        zacc[r] += a[r];
+        zacc[r] += ROPE ? Zs[n * kPitch + ti + 16 * r] : a[r];
 #pragma unroll
         for (int s = 0; s < R; ++s) acc[r][s] = fmaf(a[r], bb[s], acc[r][s]);
       }
@@ -116,14 +127,17 @@ fma_state_reduce(const float* __restrict__ partials, int P, long long E, float* 
 }
 
 // grid (ceil(N/64), units).  Thread (tn, tj) owns tokens tn + 16*r (r < 4) and outputs j = tj + 16*c.
-template <typename T, int R>
+// ROPE: the numerator uses the rotated phi(q), the denominator the plain phi(q).
+template <typename T, int R, bool ROPE>
 __global__ void __launch_bounds__(kThreads)
-fma_apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __restrict__ o, Problem p, float eps) {
+fma_apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __restrict__ o, Problem p, float eps,
+                 const float* __restrict__ cs, const float* __restrict__ sn) {
   extern __shared__ float smem[];
   const int d = p.d;
   float* Ss = smem;                     // [d][kPitch]  Ss[i][j] = S[i][j]
   float* zs = Ss + d * kPitch;          // [d]
-  float* Qs = zs + 128;                 // [kApplyTile][kPitch], phi(q)
+  float* Qs = zs + 128;                 // [kApplyTile][kPitch], phi(q) (rotated with ROPE)
+  float* Qp = Qs + kApplyTile * kPitch; // [kApplyTile][kPitch], plain phi(q) (ROPE only)
   const int u = blockIdx.y;
   const int b = u / p.H, h = u % p.H;
   const long long n0 = (long long)blockIdx.x * kApplyTile;
@@ -142,9 +156,19 @@ fma_apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __
   const long long base = (long long)b * p.sb + (long long)h * p.sh;
   for (int idx = tid; idx < kApplyTile * d; idx += kThreads) {
     const int n = idx / d, e = idx % d;
-    float x = 0.f;
-    if (n0 + n < p.N) x = fmaxf(load_f32<T>(q + base + (n0 + n) * p.sn + e), 0.f);  // phi = ReLU on the queries
+    float x = 0.f, plain = 0.f;
+    if (n0 + n < p.N) {
+      const long long off = base + (n0 + n) * p.sn + e;
+      x = plain = fmaxf(load_f32<T>(q + off), 0.f);  // phi = ReLU on the queries
+      if (ROPE && (e ^ 1) < d) {
+        const float other = fmaxf(load_f32<T>(q + off + ((e ^ 1) - e)), 0.f);
+        const long long t = (n0 + n) * (long long)(d / 2) + e / 2;
+        const float c = cs[t], sgn = sn[t];
+        x = (e & 1) ? other * sgn + plain * c : plain * c - other * sgn;
+      }
+    }
     Qs[n * kPitch + e] = x;
+    if (ROPE) Qp[n * kPitch + e] = plain;
   }
   __syncthreads();
 
@@ -165,7 +189,7 @@ fma_apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __
     for (int s = 0; s < R; ++s) bb[s] = Ss[i * kPitch + tj + 16 * s];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-      den[r] = fmaf(a[r], zz, den[r]);
+      den[r] = fmaf(ROPE ? Qp[(tn + 16 * r) * kPitch + i] : a[r], zz, den[r]);
 #pragma unroll
       for (int s = 0; s < R; ++s) acc[r][s] = fmaf(a[r], bb[s], acc[r][s]);
     }
@@ -185,21 +209,28 @@ fma_apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __
 
 template <typename T, int R>
 cudaError_t launch_state_partial(const Problem& p, const void* k, const void* v, int P, float* partials,
-                                 cudaStream_t stream) {
+                                 const float* cs, const float* sn, cudaStream_t stream) {
   dim3 grid(P, p.units());
-  fma_state_partial<T, R><<<grid, kThreads, 0, stream>>>((const T*)k, (const T*)v, p, P, partials);
+  if (cs)
+    fma_state_partial<T, R, true><<<grid, kThreads, 0, stream>>>((const T*)k, (const T*)v, p, P, partials, cs, sn);
+  else
+    fma_state_partial<T, R, false><<<grid, kThreads, 0, stream>>>((const T*)k, (const T*)v, p, P, partials, cs, sn);
   count_launches(1);
   return cudaGetLastError();
 }
 
 template <typename T, int R>
-cudaError_t launch_apply(const Problem& p, const void* q, const float* state, void* o, float eps,
-                         cudaStream_t stream) {
-  const size_t smem = sizeof(float) * ((size_t)p.d * kPitch + 128 + (size_t)kApplyTile * kPitch);
-  cudaError_t e = cudaFuncSetAttribute(fma_apply_kernel<T, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+cudaError_t launch_apply(const Problem& p, const void* q, const float* state, void* o, float eps, const float* cs,
+                         const float* sn, cudaStream_t stream) {
+  const size_t smem = sizeof(float) * ((size_t)p.d * kPitch + 128 + (size_t)(cs ? 2 : 1) * kApplyTile * kPitch);
+  cudaError_t e = cs ? cudaFuncSetAttribute(fma_apply_kernel<T, R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                     : cudaFuncSetAttribute(fma_apply_kernel<T, R, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((unsigned)((p.N + kApplyTile - 1) / kApplyTile), p.units());
-  fma_apply_kernel<T, R><<<grid, kThreads, smem, stream>>>((const T*)q, state, (T*)o, p, eps);
+  if (cs)
+    fma_apply_kernel<T, R, true><<<grid, kThreads, smem, stream>>>((const T*)q, state, (T*)o, p, eps, cs, sn);
+  else
+    fma_apply_kernel<T, R, false><<<grid, kThreads, smem, stream>>>((const T*)q, state, (T*)o, p, eps, cs, sn);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -217,33 +248,34 @@ cudaError_t launch_apply(const Problem& p, const void* q, const float* state, vo
   }
 
 cudaError_t state_partial_any(const Problem& p, const void* k, const void* v, int P, float* partials,
-                              cudaStream_t stream) {
+                              const float* cs, const float* sn, cudaStream_t stream) {
   if (p.dtype == LINATTN_F32) {
-    LINATTN_DISPATCH_R(launch_state_partial, float, p, k, v, P, partials, stream)
+    LINATTN_DISPATCH_R(launch_state_partial, float, p, k, v, P, partials, cs, sn, stream)
   } else {
-    LINATTN_DISPATCH_R(launch_state_partial, __nv_bfloat16, p, k, v, P, partials, stream)
+    LINATTN_DISPATCH_R(launch_state_partial, __nv_bfloat16, p, k, v, P, partials, cs, sn, stream)
   }
 }
 
-cudaError_t apply_any(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream) {
+cudaError_t apply_any(const Problem& p, const void* q, const float* state, void* o, float eps, const float* cs,
+                      const float* sn, cudaStream_t stream) {
   if (p.dtype == LINATTN_F32) {
-    LINATTN_DISPATCH_R(launch_apply, float, p, q, state, o, eps, stream)
+    LINATTN_DISPATCH_R(launch_apply, float, p, q, state, o, eps, cs, sn, stream)
   } else {
-    LINATTN_DISPATCH_R(launch_apply, __nv_bfloat16, p, q, state, o, eps, stream)
+    LINATTN_DISPATCH_R(launch_apply, __nv_bfloat16, p, q, state, o, eps, cs, sn, stream)
   }
 }
 
 }  // namespace
 
 cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate,
-                      float* partials, cudaStream_t stream) {
+                      float* partials, cudaStream_t stream, const float* rope_cos, const float* rope_sin) {
   const long long E = p.state_elems();
   if (p.N == 0) {
     if (accumulate) return cudaSuccess;
     return cudaMemsetAsync(state_out, 0, sizeof(float) * E * p.units(), stream);
   }
   const int P = fma_chunks(p.N);
-  cudaError_t e = state_partial_any(p, k, v, P, partials, stream);
+  cudaError_t e = state_partial_any(p, k, v, P, partials, rope_cos, rope_sin, stream);
   if (e != cudaSuccess) return e;
   dim3 grid((unsigned)((E + kThreads - 1) / kThreads), p.units());
   fma_state_reduce<<<grid, kThreads, 0, stream>>>(partials, P, E, state_out, accumulate ? 1 : 0);
@@ -251,9 +283,10 @@ cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* sta
   return cudaGetLastError();
 }
 
-cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream) {
+cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream,
+                      const float* rope_cos, const float* rope_sin) {
   if (p.N == 0) return cudaSuccess;
-  return apply_any(p, q, state, o, eps, stream);
+  return apply_any(p, q, state, o, eps, rope_cos, rope_sin, stream);
 }
 
 }  // namespace linattn

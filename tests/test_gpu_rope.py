@@ -1,0 +1,70 @@
+"""GPU parity of Eq. 2 with its rotary factors (rotation after the ReLU, numerator only) against the oracle."""
+import numpy as np
+import pytest
+
+from paper_2509_24695_b200 import synth
+from parity_util import assert_parity_bf16, assert_parity_f32, to_dev, to_f64
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-6
+
+
+@pytest.fixture(scope="module")
+def la():
+    import torch
+
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    import paper_2509_24695_b200 as la
+
+    la.load_library()
+    return la
+
+
+def gen(B, N, H, d, seed, dtype):
+    return tuple(synth.gauss((B, N, H, d), seed, t, dtype=dtype) for t in (1, 2, 3))
+
+
+SHAPES = [
+    # B, (T, Hh, Ww), H, d
+    (1, (3, 8, 8), 4, 32),
+    (2, (5, 10, 20), 3, 112),    # several tiles and a ragged tail at the paper's head dim
+    (1, (1, 1, 129), 2, 112),
+    (1, (1, 1, 1), 1, 112),
+    (1, (2, 7, 11), 2, 128),
+    (2, (3, 5, 7), 5, 64),
+    (1, (2, 5, 9), 3, 6),
+]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "B%d_T%dx%dx%d_H%d_d%d" % (s[0], *s[1], s[2], s[3]))
+def test_rope_forward_matches_oracle(la, orc, shape, dtype):
+    B, (T, Hh, Ww), H, d = shape
+    N = T * Hh * Ww
+    q, k, v = gen(B, N, H, d, 5000 + N + d, dtype)
+    cos, sin = synth.rope_table(T, Hh, Ww, d)
+    ref = orc.rope_forward(q, k, v, cos, sin, EPS)
+    o = la.linattn_forward_rope(to_dev(q), to_dev(k), to_dev(v), to_dev(cos), to_dev(sin), EPS)
+    (assert_parity_bf16 if dtype == "bf16" else assert_parity_f32)(to_f64(o), ref, f"rope forward {shape} {dtype}")
+
+
+def test_rope_with_zero_angles_is_the_plain_forward(la):
+    import torch
+
+    q, k, v = (to_dev(x) for x in gen(1, 700, 3, 112, 5100, "bf16"))
+    one = torch.ones((700, 56), dtype=torch.float32, device="cuda")
+    o = la.linattn_forward_rope(q, k, v, one, torch.zeros_like(one), EPS)
+    ref = la.linattn_forward(q, k, v, EPS)
+    # same mathematics; the two run different kernels, so compare within output rounding
+    assert_parity_bf16(to_f64(o), to_f64(ref), "zero angles")
+
+
+def test_rope_errors(la):
+    import torch
+
+    x = torch.zeros((1, 8, 2, 7), dtype=torch.bfloat16, device="cuda")
+    t = torch.zeros((8, 3), dtype=torch.float32, device="cuda")
+    with pytest.raises(la.LinAttnError) as e:
+        la.linattn_forward_rope(x, x.clone(), x.clone(), t, t.clone(), EPS)
+    assert e.value.status == -2   # odd head dim: features cannot be paired
