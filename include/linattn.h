@@ -117,15 +117,22 @@ LINATTN_API int linattn_forward(const linattn_desc* desc, int64_t N, const void*
 /* Eq. 2 as printed, with its rotary factors (Sec. 3.1): the rotation is applied after the ReLU and in the
  * numerator only,
  *     o_n = RoPE_n(phi(q_n)) ( sum_m RoPE_m(phi(k_m))^T v_m ) / ( phi(q_n) . sum_m phi(k_m) + eps ),
- * so the denominator stays non-negative.  RoPE_n turns the feature pair (2p, 2p+1) of token n by the angle
- * whose cosine and sine are rope_cos[n*(d/2) + p] and rope_sin[n*(d/2) + p]:
- * (a, b) -> (a c - b s, a s + b c).  The tables are DEVICE fp32 arrays [N][d/2], 16-byte aligned, shared by
- * all batch entries and heads; how the angles follow from a token's (t, h, w) position (the paper's 3D RoPE)
- * is the caller's choice.  d must be even.  The workspace must hold linattn_rope_workspace_bytes() bytes
- * (control block zeroed once with linattn_workspace_init). */
+ * so the denominator stays non-negative.  RoPE_n turns the feature pair (2p, 2p+1) of token n by an angle given
+ * through its cosine c and sine s: (a, b) -> (a c - b s, a s + b c).  How the angles follow from a token's
+ * (t, h, w) position (the paper's 3D RoPE) is the caller's choice.  d must be even.
+ *
+ * The rotations come as a packed DEVICE table [N][d/2] of (cos, sin) fp16 pairs (4 bytes each, 16-byte aligned
+ * base), shared by all batch entries and heads; the operation is defined on those fp16 values.  A model builds
+ * the table once (positions do not change between layers or denoising steps): linattn_rope_pack rounds fp32
+ * DEVICE arrays rope_cos, rope_sin [N][d/2] to nearest fp16 into `table` (linattn_rope_table_bytes bytes).
+ * The workspace must hold linattn_rope_workspace_bytes() bytes (control block zeroed once with
+ * linattn_workspace_init). */
+LINATTN_API int linattn_rope_table_bytes(int64_t N, int32_t d, size_t* bytes);
+LINATTN_API int linattn_rope_pack(int64_t N, int32_t d, const float* rope_cos, const float* rope_sin, void* table,
+                                  void* stream);
 LINATTN_API int linattn_rope_workspace_bytes(const linattn_desc* desc, int64_t N, size_t* bytes);
 LINATTN_API int linattn_forward_rope(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v,
-                                     void* o, float eps, const float* rope_cos, const float* rope_sin, void* workspace,
+                                     void* o, float eps, const void* rope_table, void* workspace,
                                      size_t workspace_bytes, void* stream);
 
 /* The state of Eq. 2 / Eq. 3 alone: state = (sum_n phi(k_n)^T v_n, sum_n phi(k_n)) in the layout above.

@@ -18,7 +18,7 @@ import os
 
 __all__ = [
     "LinAttnError", "library_path", "load_library", "state_bytes", "workspace_bytes", "new_workspace",
-    "linattn_forward", "linattn_forward_rope", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
+    "linattn_forward", "linattn_forward_rope", "rope_pack", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
 ]
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -70,7 +70,9 @@ def load_library(path: str | None = None):
         "linattn_workspace_status": ([vp, vp, ctypes.POINTER(ctypes.c_int)], ctypes.c_int),
         "linattn_forward": ([dp, i64, vp, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
         "linattn_rope_workspace_bytes": ([dp, i64, szp], ctypes.c_int),
-        "linattn_forward_rope": ([dp, i64, vp, vp, vp, vp, f32, vp, vp, vp, sz, vp], ctypes.c_int),
+        "linattn_rope_table_bytes": ([i64, ctypes.c_int32, szp], ctypes.c_int),
+        "linattn_rope_pack": ([i64, ctypes.c_int32, vp, vp, vp, vp], ctypes.c_int),
+        "linattn_forward_rope": ([dp, i64, vp, vp, vp, vp, f32, vp, vp, sz, vp], ctypes.c_int),
         "linattn_state": ([dp, i64, vp, vp, vp, vp, sz, vp], ctypes.c_int),
         "linattn_apply": ([dp, i64, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
         "linattn_state_static_scratch": ([dp, i64, vp, vp, vp, vp], ctypes.c_int),
@@ -178,24 +180,39 @@ def linattn_forward(q, k, v, eps: float = 1e-6, out=None, workspace=None):
     return o
 
 
-def linattn_forward_rope(q, k, v, rope_cos, rope_sin, eps: float = 1e-6, out=None, workspace=None):
-    """Eq. 2 with its rotary factors (rotation after the ReLU, numerator only).  rope_cos, rope_sin:
-    float32 CUDA tensors [N, d//2], the rotation of feature pair (2p, 2p+1) of token n."""
+def rope_pack(rope_cos, rope_sin):
+    """Packed rotary table for ``linattn_forward_rope``: float32 CUDA tensors [N, d//2] of the pair rotations'
+    cosines and sines -> one [N, d//2, 2] float16 tensor (cos, sin), rounded to nearest by the library."""
+    torch = _torch()
+    lib = load_library()
+    if rope_cos.shape != rope_sin.shape or rope_cos.dim() != 2 or rope_cos.dtype != torch.float32 or \
+            rope_sin.dtype != torch.float32 or not rope_cos.is_contiguous() or not rope_sin.is_contiguous():
+        raise ValueError("rope_cos and rope_sin must be contiguous float32 [N, d//2] tensors")
+    N, half = rope_cos.shape
+    table = torch.empty((N, half, 2), dtype=torch.float16, device=rope_cos.device)
+    _check(lib.linattn_rope_pack(N, 2 * half, _ptr(rope_cos), _ptr(rope_sin), _ptr(table), _stream(rope_cos)),
+           "linattn_rope_pack")
+    return table
+
+
+def linattn_forward_rope(q, k, v, rope_table, eps: float = 1e-6, out=None, workspace=None):
+    """Eq. 2 with its rotary factors (rotation after the ReLU, numerator only).  rope_table: the float16
+    [N, d//2, 2] (cos, sin) table of ``rope_pack``: the rotation of feature pair (2p, 2p+1) of token n."""
     torch = _torch()
     lib = load_library()
     o = torch.empty_like(q) if out is None else out
     desc = _desc_of(q, k, v, o)
     B, N, H, d = q.shape
-    for t in (rope_cos, rope_sin):
-        if tuple(t.shape) != (N, d // 2) or t.dtype != torch.float32 or not t.is_contiguous() or t.device != q.device:
-            raise ValueError("rope tables must be contiguous float32 [N, d//2] tensors on the device of q")
+    if tuple(rope_table.shape) != (N, d // 2, 2) or rope_table.dtype != torch.float16 or \
+            not rope_table.is_contiguous() or rope_table.device != q.device:
+        raise ValueError("rope_table must be a contiguous float16 [N, d//2, 2] tensor on the device of q")
     if workspace is None:
         nb = ctypes.c_size_t()
         _check(lib.linattn_rope_workspace_bytes(ctypes.byref(desc), N, ctypes.byref(nb)), "linattn_rope_workspace_bytes")
         workspace = torch.empty(nb.value, dtype=torch.uint8, device=q.device)
         _check(lib.linattn_workspace_init(_ptr(workspace), nb.value, _stream(q)), "linattn_workspace_init")
-    _check(lib.linattn_forward_rope(ctypes.byref(desc), N, _ptr(q), _ptr(k), _ptr(v), _ptr(o), eps, _ptr(rope_cos),
-                                    _ptr(rope_sin), _ptr(workspace), workspace.numel(), _stream(q)), "linattn_forward_rope")
+    _check(lib.linattn_forward_rope(ctypes.byref(desc), N, _ptr(q), _ptr(k), _ptr(v), _ptr(o), eps, _ptr(rope_table),
+                                    _ptr(workspace), workspace.numel(), _stream(q)), "linattn_forward_rope")
     return o
 
 

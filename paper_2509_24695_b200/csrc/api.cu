@@ -74,7 +74,7 @@ int cuda_status(cudaError_t e) { return e == cudaSuccess ? LINATTN_OK : LINATTN_
 int run_passes(const Problem& p, const void* k, const void* v, const void* q, void* o, float* state, bool accumulate,
                float eps, void* workspace, cudaStream_t stream, const float* base = nullptr) {
   if (umma_supported(p)) {
-    UmmaCall c{k, v, q, o, state, base, accumulate, eps};
+    UmmaCall c{k, v, q, o, state, base, accumulate, eps, nullptr};
     return umma_run(p, c, workspace, stream);
   }
   if (k && accumulate && base && base != state) {
@@ -91,6 +91,7 @@ int run_passes(const Problem& p, const void* k, const void* v, const void* q, vo
 
 // Workspace of the rotary entry point: [control block][split-N partials][one state].
 size_t rope_partial_bytes(const Problem& p) {
+  if (umma_rope_supported(p)) return umma_partial_bytes(p, true);
   return sizeof(float) * (size_t)p.state_elems() * p.units() * fma_chunks(p.N);
 }
 size_t rope_state_offset(const Problem& p) { return round256(LINATTN_WORKSPACE_CTRL_BYTES + rope_partial_bytes(p)); }
@@ -99,11 +100,14 @@ size_t rope_workspace_need(const Problem& p) { return round256(rope_state_offset
 // Eq. 2 with its rotary factors: state from the rotated keys (z from the plain ones), apply with the rotated
 // queries (denominator from the plain ones).
 int run_rope(const Problem& p, const void* q, const void* k, const void* v, void* o, float* state, float eps,
-             const float* rope_cos, const float* rope_sin, void* workspace, cudaStream_t stream) {
-  // the split-N scratch must hold the FMA path's partials too (workspace_need covers the larger of the two)
-  int st = cuda_status(fma_state(p, k, v, state, false, partials_of(workspace), stream, rope_cos, rope_sin));
+             const __half2* rope, void* workspace, cudaStream_t stream) {
+  if (umma_rope_supported(p)) {  // one launch on the tensor cores
+    UmmaCall c{k, v, q, o, state, nullptr, false, eps, rope};
+    return umma_run(p, c, workspace, stream);
+  }
+  int st = cuda_status(fma_state(p, k, v, state, false, partials_of(workspace), stream, rope));
   if (st != LINATTN_OK) return st;
-  return cuda_status(fma_apply(p, q, state, o, eps, stream, rope_cos, rope_sin));
+  return cuda_status(fma_apply(p, q, state, o, eps, stream, rope));
 }
 
 }  // namespace
@@ -301,22 +305,36 @@ int linattn_rope_workspace_bytes(const linattn_desc* desc, int64_t N, size_t* by
   return LINATTN_OK;
 }
 
+int linattn_rope_table_bytes(int64_t N, int32_t d, size_t* bytes) {
+  if (!bytes || N < 0 || d < 2) return LINATTN_ERR_INVALID_ARG;
+  if (d & 1) return LINATTN_ERR_UNSUPPORTED;
+  *bytes = (size_t)N * (size_t)(d / 2) * sizeof(__half2);
+  return LINATTN_OK;
+}
+
+int linattn_rope_pack(int64_t N, int32_t d, const float* rope_cos, const float* rope_sin, void* table, void* stream) {
+  if (N < 0 || d < 2) return LINATTN_ERR_INVALID_ARG;
+  if (d & 1) return LINATTN_ERR_UNSUPPORTED;
+  if (N > 0 && (!rope_cos || !rope_sin || !table)) return LINATTN_ERR_INVALID_ARG;
+  if (!aligned16(table)) return LINATTN_ERR_BAD_ALIGNMENT;
+  return cuda_status(rope_pack(rope_cos, rope_sin, (long long)N * (d / 2), static_cast<__half2*>(table), (cudaStream_t)stream));
+}
+
 int linattn_forward_rope(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v, void* o,
-                         float eps, const float* rope_cos, const float* rope_sin, void* workspace,
-                         size_t workspace_bytes, void* stream) {
+                         float eps, const void* rope_table, void* workspace, size_t workspace_bytes, void* stream) {
   Problem p;
   int st = resolve(desc, N, &p);
   if (st != LINATTN_OK) return st;
   if (!workspace) return LINATTN_ERR_INVALID_ARG;
   if (p.d & 1) return LINATTN_ERR_UNSUPPORTED;  // the rotation pairs features (2p, 2p+1)
-  if (N > 0 && (!q || !k || !v || !o || !rope_cos || !rope_sin || o == q || o == k || o == v))
+  if (N > 0 && (!q || !k || !v || !o || !rope_table || o == q || o == k || o == v))
     return LINATTN_ERR_INVALID_ARG;
   if ((st = check_alignment(p, q, k, v, o)) != LINATTN_OK) return st;
-  if (!aligned16(workspace) || !aligned16(rope_cos) || !aligned16(rope_sin)) return LINATTN_ERR_BAD_ALIGNMENT;
+  if (!aligned16(workspace) || !aligned16(rope_table)) return LINATTN_ERR_BAD_ALIGNMENT;
   if (workspace_bytes < rope_workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
   if (N == 0) return LINATTN_OK;
   float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + rope_state_offset(p));
-  return run_rope(p, q, k, v, o, state, eps, rope_cos, rope_sin, workspace, (cudaStream_t)stream);
+  return run_rope(p, q, k, v, o, state, eps, static_cast<const __half2*>(rope_table), workspace, (cudaStream_t)stream);
 }
 
 uint64_t linattn_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }

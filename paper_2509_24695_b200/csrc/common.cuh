@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -43,12 +44,12 @@ inline int fma_chunks(long long N) {
 
 // ---- FMA kernels (fp32 I/O path, and bf16 shapes the tensor-core kernels do not take) ----
 // state_out = (accumulate ? state_out : 0) + state of tokens [0, N); partials is scratch.
-// rope_cos / rope_sin (both or neither): Eq. 2 with its rotary factors, tables [N][d/2] of the pair rotations.
+// rope: Eq. 2 with its rotary factors, table [N][d/2] of (cos, sin) fp16 pairs, one per pair rotation.
 cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate,
-                      float* partials, cudaStream_t stream, const float* rope_cos = nullptr,
-                      const float* rope_sin = nullptr);
+                      float* partials, cudaStream_t stream, const __half2* rope = nullptr);
 cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream,
-                      const float* rope_cos = nullptr, const float* rope_sin = nullptr);
+                      const __half2* rope = nullptr);
+cudaError_t rope_pack(const float* cs, const float* sn, long long count, __half2* out, cudaStream_t stream);
 
 // ---- tensor-core (tcgen05 + TMA) kernel, bf16, d in {32 (heads contiguous), 64, 112, 128} ----
 // One launch runs the state pass (k, v non-null), the apply pass (q, o non-null), or both back to back.
@@ -61,9 +62,11 @@ struct UmmaCall {
   const float* state_base;  // `accumulate`: the reduce adds the new state to this one (may be `state` itself)
   bool accumulate;
   float eps;
+  const void* rope;  // rotary variant (Eq. 2 with its rotary factors): packed (cos, sin) fp16 table [N][d/2]; else null
 };
 bool umma_supported(const Problem& p);
-size_t umma_partial_bytes(const Problem& p);
+size_t umma_partial_bytes(const Problem& p, bool rope = false);
+bool umma_rope_supported(const Problem& p);
 // Returns LINATTN_OK or an error status.
 int umma_run(const Problem& p, const UmmaCall& call, void* workspace, cudaStream_t stream);
 

@@ -35,11 +35,11 @@ __device__ __forceinline__ void store_out<__nv_bfloat16>(__nv_bfloat16* p, float
 // grid (P, units).  R = ceil(d/16): each thread owns an R x R register tile of S:
 // rows i = ti + 16*r (key feature), columns j = tj + 16*c (value feature).
 // ROPE (Eq. 2 with its rotary factors): S is built from the rotated phi(k) (pair (2p, 2p+1) of token n turned
-// by the angle whose cosine and sine are cs[n][p], sn[n][p]), z from the plain phi(k).
+// by the angle whose (cosine, sine) is tab[n][p]), z from the plain phi(k).
 template <typename T, int R, bool ROPE>
 __global__ void __launch_bounds__(kThreads)
 fma_state_partial(const T* __restrict__ k, const T* __restrict__ v, Problem p, int P, float* __restrict__ partials,
-                  const float* __restrict__ cs, const float* __restrict__ sn) {
+                  const __half2* __restrict__ tab) {
   constexpr int kStateTile = ROPE ? 16 : 32;  // tokens staged per iteration (three staging arrays with ROPE)
   __shared__ float Ks[kStateTile * kPitch];
   __shared__ float Vs[kStateTile * kPitch];
@@ -73,8 +73,8 @@ fma_state_partial(const T* __restrict__ k, const T* __restrict__ v, Problem p, i
         vv = load_f32<T>(v + off);
         if (ROPE && (e ^ 1) < d) {  // rotate after the ReLU; an unpaired last feature stays
           const float other = fmaxf(load_f32<T>(k + off + ((e ^ 1) - e)), 0.f);
-          const long long t = (n0 + n) * (long long)(d / 2) + e / 2;
-          const float c = cs[t], sgn = sn[t];
+          const float2 cssn = __half22float2(tab[(n0 + n) * (long long)(d / 2) + e / 2]);
+          const float c = cssn.x, sgn = cssn.y;
           kv = (e & 1) ? other * sgn + kplain * c : kplain * c - other * sgn;
         }
       }
@@ -131,7 +131,7 @@ fma_state_reduce(const float* __restrict__ partials, int P, long long E, float* 
 template <typename T, int R, bool ROPE>
 __global__ void __launch_bounds__(kThreads)
 fma_apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __restrict__ o, Problem p, float eps,
-                 const float* __restrict__ cs, const float* __restrict__ sn) {
+                 const __half2* __restrict__ tab) {
   extern __shared__ float smem[];
   const int d = p.d;
   float* Ss = smem;                     // [d][kPitch]  Ss[i][j] = S[i][j]
@@ -162,8 +162,8 @@ fma_apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __
       x = plain = fmaxf(load_f32<T>(q + off), 0.f);  // phi = ReLU on the queries
       if (ROPE && (e ^ 1) < d) {
         const float other = fmaxf(load_f32<T>(q + off + ((e ^ 1) - e)), 0.f);
-        const long long t = (n0 + n) * (long long)(d / 2) + e / 2;
-        const float c = cs[t], sgn = sn[t];
+        const float2 cssn = __half22float2(tab[(n0 + n) * (long long)(d / 2) + e / 2]);
+        const float c = cssn.x, sgn = cssn.y;
         x = (e & 1) ? other * sgn + plain * c : plain * c - other * sgn;
       }
     }
@@ -209,28 +209,28 @@ fma_apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __
 
 template <typename T, int R>
 cudaError_t launch_state_partial(const Problem& p, const void* k, const void* v, int P, float* partials,
-                                 const float* cs, const float* sn, cudaStream_t stream) {
+                                 const __half2* tab, cudaStream_t stream) {
   dim3 grid(P, p.units());
-  if (cs)
-    fma_state_partial<T, R, true><<<grid, kThreads, 0, stream>>>((const T*)k, (const T*)v, p, P, partials, cs, sn);
+  if (tab)
+    fma_state_partial<T, R, true><<<grid, kThreads, 0, stream>>>((const T*)k, (const T*)v, p, P, partials, tab);
   else
-    fma_state_partial<T, R, false><<<grid, kThreads, 0, stream>>>((const T*)k, (const T*)v, p, P, partials, cs, sn);
+    fma_state_partial<T, R, false><<<grid, kThreads, 0, stream>>>((const T*)k, (const T*)v, p, P, partials, tab);
   count_launches(1);
   return cudaGetLastError();
 }
 
 template <typename T, int R>
-cudaError_t launch_apply(const Problem& p, const void* q, const float* state, void* o, float eps, const float* cs,
-                         const float* sn, cudaStream_t stream) {
-  const size_t smem = sizeof(float) * ((size_t)p.d * kPitch + 128 + (size_t)(cs ? 2 : 1) * kApplyTile * kPitch);
-  cudaError_t e = cs ? cudaFuncSetAttribute(fma_apply_kernel<T, R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+cudaError_t launch_apply(const Problem& p, const void* q, const float* state, void* o, float eps, const __half2* tab,
+                         cudaStream_t stream) {
+  const size_t smem = sizeof(float) * ((size_t)p.d * kPitch + 128 + (size_t)(tab ? 2 : 1) * kApplyTile * kPitch);
+  cudaError_t e = tab ? cudaFuncSetAttribute(fma_apply_kernel<T, R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
                      : cudaFuncSetAttribute(fma_apply_kernel<T, R, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((unsigned)((p.N + kApplyTile - 1) / kApplyTile), p.units());
-  if (cs)
-    fma_apply_kernel<T, R, true><<<grid, kThreads, smem, stream>>>((const T*)q, state, (T*)o, p, eps, cs, sn);
+  if (tab)
+    fma_apply_kernel<T, R, true><<<grid, kThreads, smem, stream>>>((const T*)q, state, (T*)o, p, eps, tab);
   else
-    fma_apply_kernel<T, R, false><<<grid, kThreads, smem, stream>>>((const T*)q, state, (T*)o, p, eps, cs, sn);
+    fma_apply_kernel<T, R, false><<<grid, kThreads, smem, stream>>>((const T*)q, state, (T*)o, p, eps, tab);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -248,34 +248,48 @@ cudaError_t launch_apply(const Problem& p, const void* q, const float* state, vo
   }
 
 cudaError_t state_partial_any(const Problem& p, const void* k, const void* v, int P, float* partials,
-                              const float* cs, const float* sn, cudaStream_t stream) {
+                              const __half2* tab, cudaStream_t stream) {
   if (p.dtype == LINATTN_F32) {
-    LINATTN_DISPATCH_R(launch_state_partial, float, p, k, v, P, partials, cs, sn, stream)
+    LINATTN_DISPATCH_R(launch_state_partial, float, p, k, v, P, partials, tab, stream)
   } else {
-    LINATTN_DISPATCH_R(launch_state_partial, __nv_bfloat16, p, k, v, P, partials, cs, sn, stream)
+    LINATTN_DISPATCH_R(launch_state_partial, __nv_bfloat16, p, k, v, P, partials, tab, stream)
   }
 }
 
-cudaError_t apply_any(const Problem& p, const void* q, const float* state, void* o, float eps, const float* cs,
-                      const float* sn, cudaStream_t stream) {
+cudaError_t apply_any(const Problem& p, const void* q, const float* state, void* o, float eps, const __half2* tab,
+                      cudaStream_t stream) {
   if (p.dtype == LINATTN_F32) {
-    LINATTN_DISPATCH_R(launch_apply, float, p, q, state, o, eps, cs, sn, stream)
+    LINATTN_DISPATCH_R(launch_apply, float, p, q, state, o, eps, tab, stream)
   } else {
-    LINATTN_DISPATCH_R(launch_apply, __nv_bfloat16, p, q, state, o, eps, cs, sn, stream)
+    LINATTN_DISPATCH_R(launch_apply, __nv_bfloat16, p, q, state, o, eps, tab, stream)
   }
+}
+
+// (cos, sin) of every pair rotation as one fp16 pair, round to nearest.
+__global__ void rope_pack_kernel(const float* __restrict__ cs, const float* __restrict__ sn, long long count,
+                                 __half2* __restrict__ out) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) out[i] = __floats2half2_rn(cs[i], sn[i]);
 }
 
 }  // namespace
 
+cudaError_t rope_pack(const float* cs, const float* sn, long long count, __half2* out, cudaStream_t stream) {
+  if (count == 0) return cudaSuccess;
+  rope_pack_kernel<<<(unsigned)((count + 255) / 256), 256, 0, stream>>>(cs, sn, count, out);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
 cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* state_out, bool accumulate,
-                      float* partials, cudaStream_t stream, const float* rope_cos, const float* rope_sin) {
+                      float* partials, cudaStream_t stream, const __half2* rope) {
   const long long E = p.state_elems();
   if (p.N == 0) {
     if (accumulate) return cudaSuccess;
     return cudaMemsetAsync(state_out, 0, sizeof(float) * E * p.units(), stream);
   }
   const int P = fma_chunks(p.N);
-  cudaError_t e = state_partial_any(p, k, v, P, partials, rope_cos, rope_sin, stream);
+  cudaError_t e = state_partial_any(p, k, v, P, partials, rope, stream);
   if (e != cudaSuccess) return e;
   dim3 grid((unsigned)((E + kThreads - 1) / kThreads), p.units());
   fma_state_reduce<<<grid, kThreads, 0, stream>>>(partials, P, E, state_out, accumulate ? 1 : 0);
@@ -284,9 +298,9 @@ cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* sta
 }
 
 cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream,
-                      const float* rope_cos, const float* rope_sin) {
+                      const __half2* rope) {
   if (p.N == 0) return cudaSuccess;
-  return apply_any(p, q, state, o, eps, rope_cos, rope_sin, stream);
+  return apply_any(p, q, state, o, eps, rope, stream);
 }
 
 }  // namespace linattn

@@ -175,7 +175,11 @@ struct FusedParams {
   float* partials;         // one record of G head-states per (CTA, unit) segment of the state pass
   float eps;
   WorkspaceCtrl* ctrl;
+  const uint4* rope;       // rotary variant: [N][d/8] chunks of four (cos, sin) fp16 pairs; null otherwise
+  long long N;             // tokens (bound of the rotary table)
 };
+
+constexpr int kZParts = 4 * 128;  // rotary variant: floats a partial record carries for z (per ReLU warp, per feature)
 
 // TMA coordinates (feature, head) of 64-element box `box` (0/1) of head group hg
 template <int D>
@@ -218,6 +222,28 @@ __device__ __forceinline__ void relu_pass(uint8_t* box0, uint8_t* box1, int t) {
     }
   }
 }
+
+// Rotary variant: a 16-byte chunk holds four feature pairs; `tab` holds their (cos, sin) as fp16 pairs.
+// (a, b) -> (a c - b s, a s + b c), rounded to bf16.
+__device__ __forceinline__ void unpack_relu8(const uint4& x, float (&f)[8]) {
+  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    f[2 * e] = fmaxf(__uint_as_float(w[e] << 16), 0.f);
+    f[2 * e + 1] = fmaxf(__uint_as_float(w[e] & 0xFFFF0000u), 0.f);
+  }
+}
+__device__ __forceinline__ uint4 rotate_pack8(const float (&f)[8], const uint4& tab) {
+  const uint32_t t[4] = {tab.x, tab.y, tab.z, tab.w};
+  uint32_t o[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 cs = __half22float2(*reinterpret_cast<const __half2*>(&t[e]));
+    o[e] = pack_bf16x2(f[2 * e] * cs.x - f[2 * e + 1] * cs.y, f[2 * e] * cs.y + f[2 * e + 1] * cs.x);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+constexpr uint32_t kRopeIdentity = 0x00003C00u;  // (cos, sin) = (1, 0) as an fp16 pair
 
 // ---------------------------------------------------------------- grid barrier
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
@@ -264,11 +290,11 @@ __device__ __forceinline__ int trailing_cta_of(long long f, long long tot, int R
 
 __device__ __forceinline__ void add4(float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
 
-template <int D>
+template <int D, bool ROPE>
 __device__ void reduce_slice(const FusedParams& p) {
   using C = Cfg<D>;
   constexpr int E4 = (D + 1) * D / 4;  // float4 per head state
-  constexpr int REC4 = C::G * E4;      // float4 per partial record
+  constexpr int REC4 = C::G * E4 + (ROPE ? kZParts / 4 : 0);  // float4 per partial record
   const Sched& s = p.sa;
   const long long tot = (long long)p.B * p.H * E4;
   const long long i0 = (long long)blockIdx.x * tot / gridDim.x;
@@ -290,6 +316,21 @@ __device__ void reduce_slice(const FusedParams& p) {
       ntrail = trailing_cta_of((long long)(u + 1) * s.m - 1, ttot, s.R) - r_lo + 1;
     }
     const int nrec = ncol + ntrail;
+    if (ROPE && e >= D * D / 4) {
+      // rotary variant: z comes from the plain phi(k) sums that the four ReLU warps of every segment left
+      // behind the record (per warp, per feature); records in their fixed order, warps 0..3 within each
+      const float4* zp = reinterpret_cast<const float4*>(p.partials) + E4 + (e - D * D / 4);
+      for (int kk = 0; kk < nrec; ++kk) {
+        const int rec = kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u;
+        float4 w4[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) w4[w] = __ldcg(zp + (size_t)rec * REC4 + w * 32);
+#pragma unroll
+        for (int w = 0; w < 4; ++w) add4(sum, w4[w]);
+      }
+      state4[idx] = sum;
+      continue;
+    }
     for (int k0 = 0; k0 < nrec; k0 += 12) {
       float4 v[12];
 #pragma unroll
@@ -362,7 +403,7 @@ __device__ __forceinline__ void build_s_operand(uint8_t* s_op, const float* __re
 }
 
 // ============================================================================ the kernel
-template <int D>
+template <int D, bool ROPE>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                   const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o, FusedParams p) {
@@ -513,10 +554,75 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     // ------------------------------------------------------------ ReLU pass over the K boxes
     const int tr = threadIdx.x - kReluThread0;
     uint32_t it = 0;
+    // rotary variant: this thread's 16-byte column holds logical chunk lc of every row it touches
+    const int row0 = tr >> 3, pc = tr & 7, lc = pc ^ (row0 & 7);
+    const bool box1_live = 64 + lc * 8 < C::FEAT;
+    float zacc[16];  // sums of the plain phi(k) over the segment: features 8*lc.. of box 0, 64 + 8*lc.. of box 1
+#pragma unroll
+    for (int e = 0; e < 16; ++e) zacc[e] = 0.f;
     for (TileWalk t(wa); !t.done(); t.next(), ++it) {
       const int s = it % NSA;
-      if (!mbar_wait(&a_full[s], (it / NSA) & 1, abort_flag)) break;
       uint8_t* st = smem + s * STAGE;
+      if (ROPE) {
+        // the rotations of this stage's rows do not depend on K: ask for them before waiting for the tile
+        uint4 tab0[kTileState / 16], tab1[kTileState / 16];
+#pragma unroll
+        for (int i = 0; i < kTileState / 16; ++i) {
+          const long long n = (long long)t.tile() * kTileState + row0 + 16 * i;
+          tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
+          if (n < p.N) {
+            tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
+            if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
+          }
+        }
+        if (!__all_sync(0xffffffffu, mbar_wait(&a_full[s], (it / NSA) & 1, abort_flag))) break;  // leave as a whole warp
+        uint8_t* p0 = st + C::KOFF + row0 * kRowBytes + pc * 16;
+#pragma unroll
+        for (int i = 0; i < kTileState / 16; ++i) {
+          float f[8];
+          uint4* c0 = reinterpret_cast<uint4*>(p0 + i * 16 * kRowBytes);
+          unpack_relu8(*c0, f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) zacc[e] += f[e];
+          *c0 = rotate_pack8(f, tab0[i]);
+          if (box1_live) {
+            uint4* c1 = reinterpret_cast<uint4*>(p0 + kBox + i * 16 * kRowBytes);
+            unpack_relu8(*c1, f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) zacc[8 + e] += f[e];
+            *c1 = rotate_pack8(f, tab1[i]);
+          }
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(&a_ready[s]);
+        if (t.seg_last()) {
+          // leave the segment's sums behind the record: the four lanes of this warp that share a chunk add
+          // up in a fixed order, then one of them stores
+          const int w = tr >> 5, r = (tr >> 3) & 3;
+          float tot[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) tot[e] = 0.f;
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) {
+            const int src = (rr << 3) | (lc ^ ((4 * (w & 1) + rr) & 7));
+#pragma unroll
+            for (int e = 0; e < 16; ++e) tot[e] += __shfl_sync(0xffffffffu, zacc[e], src);
+          }
+          if (r == 0) {
+            float* zp = p.partials + (size_t)t.record() * (C::G * (D + 1) * D + kZParts) + C::G * (D + 1) * D + w * 128;
+            *reinterpret_cast<float4*>(zp + 8 * lc) = make_float4(tot[0], tot[1], tot[2], tot[3]);
+            *reinterpret_cast<float4*>(zp + 8 * lc + 4) = make_float4(tot[4], tot[5], tot[6], tot[7]);
+            if (box1_live) {
+              *reinterpret_cast<float4*>(zp + 64 + 8 * lc) = make_float4(tot[8], tot[9], tot[10], tot[11]);
+              *reinterpret_cast<float4*>(zp + 64 + 8 * lc + 4) = make_float4(tot[12], tot[13], tot[14], tot[15]);
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 16; ++e) zacc[e] = 0.f;
+        }
+        continue;
+      }
+      if (!mbar_wait(&a_full[s], (it / NSA) & 1, abort_flag)) break;
       relu_pass<C::FEAT, kTileState>(st + C::KOFF, st + C::KOFF + kBox, tr);
       if (!C::ONES_BOX && tr < kTileState) {
         // value column 112 := 1 (logical chunk 6 of the second V box, element 0), so z is accumulator column 112
@@ -541,7 +647,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       const int h = hg * C::G + g;
       const bool live = i < C::FEAT && h < p.H;
       // record of this (CTA, unit) segment: G consecutive head-states in the library's layout
-      float* out = p.partials + ((size_t)t.record() * C::G + g) * ((size_t)(D + 1) * D);
+      float* out = p.partials + (size_t)t.record() * (C::G * (D + 1) * D + (ROPE ? kZParts : 0)) + (size_t)g * ((D + 1) * D);
       const uint32_t trow = tmem_base + ((uint32_t)(wq * 32) << 16);
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
@@ -568,7 +674,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
             const int j = cc * 32 + x;             // value feature within the group
             const int jl = j - g * D;
             if (jl >= 0 && jl < D) out[(size_t)jl * D + il] = sum[x];
-            if (!C::ONES_BOX && j == C::ZCOL) out[(size_t)D * D + il] = sum[x];
+            if (!C::ONES_BOX && !ROPE && j == C::ZCOL) out[(size_t)D * D + il] = sum[x];  // (rotary: z comes from the ReLU warps)
           }
         }
       }
@@ -592,7 +698,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   // ==================================================================== reduce
   if (p.do_state) {
     grid_barrier(p.ctrl, abort_flag);
-    if (!*abort_flag) reduce_slice<D>(p);
+    if (!*abort_flag) reduce_slice<D, ROPE>(p);
     if (p.do_apply) grid_barrier(p.ctrl, abort_flag);
   }
   if (C::G > 1 && wc.f1 > wc.f0) {
@@ -643,6 +749,12 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     const int tr = threadIdx.x - kReluThread0;
     uint32_t it = 0, seg = 0;
     bool ok = true;
+    // rotary variant: this thread's 16-byte column holds logical chunk lc of every row it touches
+    const int row0 = tr >> 3, pc = tr & 7, lc = pc ^ (row0 & 7);
+    const bool box1_live = 64 + lc * 8 < C::FEAT;
+    float zc[16];  // the segment's z at this thread's features (8*lc.. of box 0, 64 + 8*lc.. of box 1)
+#pragma unroll
+    for (int e = 0; e < 16; ++e) zc[e] = 0.f;
     for (TileWalk t(wc); !t.done() && ok; t.next(), ++it) {
       const int s = it % NSC;
       if (t.seg_first()) {
@@ -651,9 +763,59 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         if (!ok) break;
         const int u = t.unit();
         build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, tr, 256);
+        if (ROPE) {
+          const float4* zrow = reinterpret_cast<const float4*>(p.state + ((size_t)u * (D + 1) + D) * D);  // G = 1: unit = (b, h)
+          const float4 a0 = __ldcg(zrow + 2 * lc), a1 = __ldcg(zrow + 2 * lc + 1);
+          zc[0] = a0.x; zc[1] = a0.y; zc[2] = a0.z; zc[3] = a0.w; zc[4] = a1.x; zc[5] = a1.y; zc[6] = a1.z; zc[7] = a1.w;
+          if (box1_live) {
+            const float4 b0 = __ldcg(zrow + 16 + 2 * lc), b1 = __ldcg(zrow + 16 + 2 * lc + 1);
+            zc[8] = b0.x; zc[9] = b0.y; zc[10] = b0.z; zc[11] = b0.w; zc[12] = b1.x; zc[13] = b1.y; zc[14] = b1.z; zc[15] = b1.w;
+          }
+        }
         fence_proxy_async_smem();
         mbar_arrive(s_ready);
         ++seg;
+      }
+      if (ROPE) {
+        // numerator operand: rotated phi(q); denominator: plain phi(q) . z, added up over the eight lanes that
+        // share a row and left in the row's zero padding (features 112..) for the epilogue
+        uint8_t* sl = slots + s * SLOT;
+        uint4 tab0[kTileApply / 16], tab1[kTileApply / 16];
+#pragma unroll
+        for (int i = 0; i < kTileApply / 16; ++i) {
+          const long long n = (long long)t.tile() * kTileApply + row0 + 16 * i;
+          tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
+          if (n < p.N) {
+            tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
+            if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
+          }
+        }
+        if (!__all_sync(0xffffffffu, mbar_wait(&c_full[s], (it / NSC) & 1, abort_flag))) break;  // leave as a whole warp
+        uint8_t* p0 = sl + row0 * kRowBytes + pc * 16;
+#pragma unroll
+        for (int i = 0; i < kTileApply / 16; ++i) {
+          float f[8];
+          uint4* c0 = reinterpret_cast<uint4*>(p0 + i * 16 * kRowBytes);
+          unpack_relu8(*c0, f);
+          float den = 0.f;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) den = fmaf(f[e], zc[e], den);
+          *c0 = rotate_pack8(f, tab0[i]);
+          uint4* c1 = reinterpret_cast<uint4*>(p0 + HALF + i * 16 * kRowBytes);
+          if (box1_live) {
+            unpack_relu8(*c1, f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) den = fmaf(f[e], zc[8 + e], den);
+            *c1 = rotate_pack8(f, tab1[i]);
+          }
+          den += __shfl_xor_sync(0xffffffffu, den, 1);
+          den += __shfl_xor_sync(0xffffffffu, den, 2);
+          den += __shfl_xor_sync(0xffffffffu, den, 4);
+          if (lc == 6) *reinterpret_cast<float*>(c1) = den;  // chunk 6 of the second box: features 112..119
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(&c_ready[s]);
+        continue;
       }
       if (!mbar_wait(&c_full[s], (it / NSC) & 1, abort_flag)) break;
       relu_pass<C::FEAT, kTileApply>(slots + s * SLOT, slots + s * SLOT + HALF, tr);
@@ -682,13 +844,19 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       tcgen05_fence_after();
       if (t.seg_last()) mbar_arrive(seg_done);
       const uint32_t trow = tmem_base + acc * kAccStride + ((uint32_t)(wq * 32) << 16);
-      uint32_t dn[4];
-      tmem_ld_x4(trow + C::ZROW, dn);
-      tmem_ld_wait();
-      float rinv[C::G];
-#pragma unroll
-      for (int g = 0; g < C::G; ++g) rinv[g] = 1.0f / (__uint_as_float(dn[g]) + p.eps);  // eps added once, after the dot product
       uint8_t* sl = slots + s * SLOT;
+      float rinv[C::G];
+      if (ROPE) {
+        // the ReLU warps left phi(q) . z of this row in the row's padding
+        const float den = *reinterpret_cast<const float*>(sl + HALF + r * kRowBytes + ((6 ^ (r & 7)) << 4));
+        rinv[0] = 1.0f / (den + p.eps);
+      } else {
+        uint32_t dn[4];
+        tmem_ld_x4(trow + C::ZROW, dn);
+        tmem_ld_wait();
+#pragma unroll
+        for (int g = 0; g < C::G; ++g) rinv[g] = 1.0f / (__uint_as_float(dn[g]) + p.eps);  // eps added once, after the dot product
+      }
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
         if (cc * 32 >= C::FEAT) break;
@@ -812,7 +980,7 @@ int sm_count() {
 
 inline int groups_of(int d) { return d == 32 ? 4 : d == 64 ? 2 : 1; }
 
-template <int D>
+template <int D, bool ROPE>
 int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
   using C = Cfg<D>;
   const int sms = sm_count();
@@ -829,6 +997,8 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   fp.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + LINATTN_WORKSPACE_CTRL_BYTES);
   fp.eps = c.eps;
   fp.ctrl = static_cast<WorkspaceCtrl*>(workspace);
+  fp.rope = static_cast<const uint4*>(c.rope);
+  fp.N = p.N;
   int grid = 0;
   if (do_state) grid = fp.sa.grid;
   if (do_apply && fp.sc.grid > grid) grid = fp.sc.grid;
@@ -846,13 +1016,13 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   if (!do_state) { mk = mq; mv = mq; }
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(umma_fused_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM) !=
+    if (cudaFuncSetAttribute(umma_fused_kernel<D, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM) !=
         cudaSuccess)
       return LINATTN_ERR_CUDA;
     attr_set = true;
   }
   void* args[] = {&mk, &mv, &mq, &mo, &fp};
-  const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D>, dim3(grid), dim3(kThreads), args,
+  const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D, ROPE>, dim3(grid), dim3(kThreads), args,
                                                     C::SMEM, stream);
   if (e != cudaSuccess) { cudaGetLastError(); return LINATTN_ERR_CUDA; }
   count_launches(1);
@@ -868,19 +1038,23 @@ bool umma_supported(const Problem& p) {
 }
 
 // One partial record (G head-states) per (CTA, unit) segment of the state pass: at most kMaxCtas + units.
-size_t umma_partial_bytes(const Problem& p) {
+size_t umma_partial_bytes(const Problem& p, bool rope) {
   const int G = groups_of(p.d);
   const size_t units = (size_t)p.B * ((p.H + G - 1) / G);
-  return ((size_t)kMaxCtas + units) * G * (size_t)p.state_elems() * sizeof(float);
+  return ((size_t)kMaxCtas + units) * (G * (size_t)p.state_elems() + (rope ? kZParts : 0)) * sizeof(float);
 }
+
+// The rotary variant runs on the tensor cores at the paper's head dim (the denominators travel in the zero
+// padding of the 112-feature rows); other shapes take the FMA kernels.
+bool umma_rope_supported(const Problem& p) { return umma_supported(p) && p.d == 112; }
 
 int umma_run(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
   if (p.N == 0 || (!c.k && !c.q)) return LINATTN_OK;
   switch (p.d) {
-    case 32: return launch_fused<32>(p, c, workspace, stream);
-    case 64: return launch_fused<64>(p, c, workspace, stream);
-    case 112: return launch_fused<112>(p, c, workspace, stream);
-    case 128: return launch_fused<128>(p, c, workspace, stream);
+    case 32: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<32, false>(p, c, workspace, stream);
+    case 64: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<64, false>(p, c, workspace, stream);
+    case 112: return c.rope ? launch_fused<112, true>(p, c, workspace, stream) : launch_fused<112, false>(p, c, workspace, stream);
+    case 128: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<128, false>(p, c, workspace, stream);
   }
   return LINATTN_ERR_UNSUPPORTED;
 }

@@ -114,3 +114,19 @@ def test_720p_stream_eighty_steps(la, orc):
     ref = orc.apply_rows(q_last, S, z, w.eps, rows)
     assert_parity_bf16(to_f64(out[:, torch.from_numpy(rows).cuda()]), ref, "last step sampled rows")
     assert la.workspace_status(cache.workspace) == 0
+
+
+def test_480p_layer_with_rotary_factors(la, orc):
+    """Eq. 2 with its rotary factors at the 480p size (21 x 30 x 52 tokens, a 3D table), every output row."""
+    import torch
+
+    w = synth.P480
+    q, k, v = synth.qkv(w)
+    cos, sin = synth.rope_table(21, 30, 52, w.d)
+    table = la.rope_pack(to_dev(cos), to_dev(sin))
+    packed = table.cpu().numpy().astype(np.float64)
+    o = la.linattn_forward_rope(to_dev(q), to_dev(k), to_dev(v), table, w.eps)
+    o2 = la.linattn_forward_rope(to_dev(q), to_dev(k), to_dev(v), table, w.eps)
+    assert torch.equal(o, o2)  # run-to-run determinism
+    ref = orc.rope_forward(q, k, v, packed[..., 0], packed[..., 1], w.eps)
+    assert_parity_bf16(to_f64(o), ref, "480p rotary")

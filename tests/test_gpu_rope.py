@@ -44,8 +44,13 @@ def test_rope_forward_matches_oracle(la, orc, shape, dtype):
     N = T * Hh * Ww
     q, k, v = gen(B, N, H, d, 5000 + N + d, dtype)
     cos, sin = synth.rope_table(T, Hh, Ww, d)
-    ref = orc.rope_forward(q, k, v, cos, sin, EPS)
-    o = la.linattn_forward_rope(to_dev(q), to_dev(k), to_dev(v), to_dev(cos), to_dev(sin), EPS)
+    table = la.rope_pack(to_dev(cos), to_dev(sin))
+    # the operation is defined on the packed fp16 (cos, sin) values: the oracle gets exactly those
+    packed = table.cpu().numpy().astype(np.float64)
+    assert np.array_equal(packed[..., 0], cos.astype(np.float16).astype(np.float64))
+    assert np.array_equal(packed[..., 1], sin.astype(np.float16).astype(np.float64))
+    ref = orc.rope_forward(q, k, v, packed[..., 0], packed[..., 1], EPS)
+    o = la.linattn_forward_rope(to_dev(q), to_dev(k), to_dev(v), table, EPS)
     (assert_parity_bf16 if dtype == "bf16" else assert_parity_f32)(to_f64(o), ref, f"rope forward {shape} {dtype}")
 
 
@@ -54,7 +59,7 @@ def test_rope_with_zero_angles_is_the_plain_forward(la):
 
     q, k, v = (to_dev(x) for x in gen(1, 700, 3, 112, 5100, "bf16"))
     one = torch.ones((700, 56), dtype=torch.float32, device="cuda")
-    o = la.linattn_forward_rope(q, k, v, one, torch.zeros_like(one), EPS)
+    o = la.linattn_forward_rope(q, k, v, la.rope_pack(one, torch.zeros_like(one)), EPS)
     ref = la.linattn_forward(q, k, v, EPS)
     # same mathematics; the two run different kernels, so compare within output rounding
     assert_parity_bf16(to_f64(o), to_f64(ref), "zero angles")
@@ -64,7 +69,7 @@ def test_rope_errors(la):
     import torch
 
     x = torch.zeros((1, 8, 2, 7), dtype=torch.bfloat16, device="cuda")
-    t = torch.zeros((8, 3), dtype=torch.float32, device="cuda")
+    t = torch.zeros((8, 3, 2), dtype=torch.float16, device="cuda")
     with pytest.raises(la.LinAttnError) as e:
-        la.linattn_forward_rope(x, x.clone(), x.clone(), t, t.clone(), EPS)
+        la.linattn_forward_rope(x, x.clone(), x.clone(), t, EPS)
     assert e.value.status == -2   # odd head dim: features cannot be paired
