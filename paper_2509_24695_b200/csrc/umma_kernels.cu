@@ -40,10 +40,19 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 352;
-constexpr int kReluThread0 = 64;    // warps 2-5
-constexpr int kEpiThread0 = 192;    // warps 6-9
-constexpr int kStoreWarp = 10;
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, then the ReLU warps, four epilogue warps, one store
+// warp.  The rotary variant does several times the arithmetic per element in the ReLU role (rotation,
+// sums for z, denominators), so it runs that role on eight warps instead of four.
+template <bool ROPE>
+struct Roles {
+  static constexpr int RELU_WARPS = ROPE ? 8 : 4;
+  static constexpr int RELU_THREADS = RELU_WARPS * 32;
+  static constexpr int EPI_WARP0 = 2 + RELU_WARPS;
+  static constexpr int EPI_THREAD0 = EPI_WARP0 * 32;
+  static constexpr int STORE_WARP = EPI_WARP0 + 4;
+  static constexpr int THREADS = (STORE_WARP + 1) * 32;
+};
+constexpr int kReluThread0 = 64;
 constexpr int kTileApply = 128;     // tokens per apply tile (= UMMA M)
 constexpr int kTileState = 64;      // tokens per state stage (4 UMMA K steps of 16 tokens)
 constexpr int kRowBytes = 128;      // one swizzle row: 64 bf16
@@ -179,7 +188,7 @@ struct FusedParams {
   long long N;             // tokens (bound of the rotary table)
 };
 
-constexpr int kZParts = 4 * 128;  // rotary variant: floats a partial record carries for z (per ReLU warp, per feature)
+constexpr int kZParts = 8 * 128;  // rotary variant: floats a partial record carries for z (per ReLU warp, per feature)
 
 // TMA coordinates (feature, head) of 64-element box `box` (0/1) of head group hg
 template <int D>
@@ -302,7 +311,7 @@ __device__ void reduce_slice(const FusedParams& p) {
   const int ncol = s.P == 0 ? 0 : (s.P < (s.tpu + s.Lc - 1) / s.Lc ? s.P : (s.tpu + s.Lc - 1) / s.Lc);
   const long long ttot = (long long)s.U * s.m;
   float4* state4 = reinterpret_cast<float4*>(p.state);
-  for (long long idx = i0 + threadIdx.x; idx < i1; idx += kThreads) {
+  for (long long idx = i0 + threadIdx.x; idx < i1; idx += blockDim.x) {
     const int bh = (int)(idx / E4), e = (int)(idx % E4);
     const int b = bh / p.H, h = bh % p.H;
     const int u = b * p.HG + h / C::G, g = h % C::G;
@@ -318,15 +327,15 @@ __device__ void reduce_slice(const FusedParams& p) {
     const int nrec = ncol + ntrail;
     if (ROPE && e >= D * D / 4) {
       // rotary variant: z comes from the plain phi(k) sums that the four ReLU warps of every segment left
-      // behind the record (per warp, per feature); records in their fixed order, warps 0..3 within each
+      // behind the record (per warp, per feature); records in their fixed order, warps 0..7 within each
       const float4* zp = reinterpret_cast<const float4*>(p.partials) + E4 + (e - D * D / 4);
       for (int kk = 0; kk < nrec; ++kk) {
         const int rec = kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u;
-        float4 w4[4];
+        float4 w4[8];
 #pragma unroll
-        for (int w = 0; w < 4; ++w) w4[w] = __ldcg(zp + (size_t)rec * REC4 + w * 32);
+        for (int w = 0; w < 8; ++w) w4[w] = __ldcg(zp + (size_t)rec * REC4 + w * 32);
 #pragma unroll
-        for (int w = 0; w < 4; ++w) add4(sum, w4[w]);
+        for (int w = 0; w < 8; ++w) add4(sum, w4[w]);
       }
       state4[idx] = sum;
       continue;
@@ -404,10 +413,11 @@ __device__ __forceinline__ void build_s_operand(uint8_t* s_op, const float* __re
 
 // ============================================================================ the kernel
 template <int D, bool ROPE>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(Roles<ROPE>::THREADS, 1)
 umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                   const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o, FusedParams p) {
   using C = Cfg<D>;
+  using R = Roles<ROPE>;
   constexpr int NSA = C::STATE_STAGES;
   constexpr int STAGE = C::STAGE_BYTES;
   constexpr int NSC = C::APPLY_SLOTS;
@@ -445,15 +455,15 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   const Work wc = p.do_apply ? work_of(p.sc, blockIdx.x) : work_of(p.sc, 0x7fffffff);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NSA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_ready[s], 128); mbar_init(&a_empty[s], 1); }
+    for (int s = 0; s < NSA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_ready[s], R::RELU_THREADS); mbar_init(&a_empty[s], 1); }
     mbar_init(a_tfull, 1);
     mbar_init(a_tempty, 128);
     mbar_init(a_done, 1);
     for (int s = 0; s < NSC; ++s) {
-      mbar_init(&c_full[s], 1); mbar_init(&c_ready[s], 128); mbar_init(&c_empty[s], 1); mbar_init(&c_staged[s], 128);
+      mbar_init(&c_full[s], 1); mbar_init(&c_ready[s], R::RELU_THREADS); mbar_init(&c_empty[s], 1); mbar_init(&c_staged[s], 128);
     }
     for (int b = 0; b < 2; ++b) { mbar_init(&c_tfull[b], 1); mbar_init(&c_tempty[b], 128); }
-    mbar_init(s_ready, 256);
+    mbar_init(s_ready, R::RELU_THREADS + 128);
     mbar_init(seg_done, 128);
     *abort_flag = 0;
     fence_mbar_init();
@@ -464,7 +474,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   }
   if (C::ONES_BOX && wa.f1 > wa.f0) {
     // the constant "ones" chunk of every stage: value columns 128..191 of B, of which column 128 is 1
-    for (int idx = threadIdx.x; idx < NSA * (kBox / 16); idx += kThreads) {
+    for (int idx = threadIdx.x; idx < NSA * (kBox / 16); idx += R::THREADS) {
       const int s = idx / (kBox / 16), c = idx % (kBox / 16);
       const int row = c >> 3, phys = c & 7;
       uint4 val = make_uint4(0, 0, 0, 0);
@@ -550,7 +560,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       }
       if (it > 0) umma_commit(a_done); else mbar_arrive(a_done);
     }
-  } else if (warp < 6) {
+  } else if (warp < R::EPI_WARP0) {
     // ------------------------------------------------------------ ReLU pass over the K boxes
     const int tr = threadIdx.x - kReluThread0;
     uint32_t it = 0;
@@ -560,38 +570,48 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     float zacc[16];  // sums of the plain phi(k) over the segment: features 8*lc.. of box 0, 64 + 8*lc.. of box 1
 #pragma unroll
     for (int e = 0; e < 16; ++e) zacc[e] = 0.f;
+    // The rotations of a row do not depend on K: they are fetched one stage ahead, each register reloaded
+    // for the next stage right after its use, so that their latency is off the stage's critical path.
+    uint4 tab0[kTileState / 32], tab1[kTileState / 32];
+    auto fetch_rot = [&](int tile, int i) {
+      const long long n = (long long)tile * kTileState + row0 + 32 * i;
+      tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
+      if (n < p.N) {
+        tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
+        if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
+      }
+    };
+    if (ROPE) {
+      TileWalk t0(wa);
+      if (!t0.done()) {
+#pragma unroll
+        for (int i = 0; i < kTileState / 32; ++i) fetch_rot(t0.tile(), i);
+      }
+    }
     for (TileWalk t(wa); !t.done(); t.next(), ++it) {
       const int s = it % NSA;
       uint8_t* st = smem + s * STAGE;
       if (ROPE) {
-        // the rotations of this stage's rows do not depend on K: ask for them before waiting for the tile
-        uint4 tab0[kTileState / 16], tab1[kTileState / 16];
-#pragma unroll
-        for (int i = 0; i < kTileState / 16; ++i) {
-          const long long n = (long long)t.tile() * kTileState + row0 + 16 * i;
-          tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
-          if (n < p.N) {
-            tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
-            if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
-          }
-        }
+        TileWalk tn = t;
+        tn.next();
         if (!__all_sync(0xffffffffu, mbar_wait(&a_full[s], (it / NSA) & 1, abort_flag))) break;  // leave as a whole warp
         uint8_t* p0 = st + C::KOFF + row0 * kRowBytes + pc * 16;
 #pragma unroll
-        for (int i = 0; i < kTileState / 16; ++i) {
+        for (int i = 0; i < kTileState / 32; ++i) {
           float f[8];
-          uint4* c0 = reinterpret_cast<uint4*>(p0 + i * 16 * kRowBytes);
+          uint4* c0 = reinterpret_cast<uint4*>(p0 + i * 32 * kRowBytes);
           unpack_relu8(*c0, f);
 #pragma unroll
           for (int e = 0; e < 8; ++e) zacc[e] += f[e];
           *c0 = rotate_pack8(f, tab0[i]);
           if (box1_live) {
-            uint4* c1 = reinterpret_cast<uint4*>(p0 + kBox + i * 16 * kRowBytes);
+            uint4* c1 = reinterpret_cast<uint4*>(p0 + kBox + i * 32 * kRowBytes);
             unpack_relu8(*c1, f);
 #pragma unroll
             for (int e = 0; e < 8; ++e) zacc[8 + e] += f[e];
             *c1 = rotate_pack8(f, tab1[i]);
           }
+          if (!tn.done()) fetch_rot(tn.tile(), i);
         }
         fence_proxy_async_smem();
         mbar_arrive(&a_ready[s]);
@@ -631,7 +651,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       fence_proxy_async_smem();
       mbar_arrive(&a_ready[s]);
     }
-  } else if (warp < kStoreWarp) {
+  } else if (warp < R::STORE_WARP) {
     // ------------------------------------------------------------ epilogue: accumulator -> partial record
     const int wq = warp & 3;
     const int i = wq * 32 + lane;           // accumulator lane = key feature within the group
@@ -703,7 +723,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   }
   if (C::G > 1 && wc.f1 > wc.f0) {
     // cross-head blocks of the packed S operand are never written by a head: they must read as zero
-    for (int idx = threadIdx.x; idx < C::S_BYTES / 16; idx += kThreads)
+    for (int idx = threadIdx.x; idx < C::S_BYTES / 16; idx += R::THREADS)
       *reinterpret_cast<uint4*>(s_op + idx * 16) = make_uint4(0, 0, 0, 0);
     __syncthreads();
   }
@@ -744,7 +764,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         umma_commit(&c_tfull[acc]);
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < R::EPI_WARP0) {
     // ------------------------------------------------------------ ReLU pass over Q tiles (+ half of the S build)
     const int tr = threadIdx.x - kReluThread0;
     uint32_t it = 0, seg = 0;
@@ -755,6 +775,23 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     float zc[16];  // the segment's z at this thread's features (8*lc.. of box 0, 64 + 8*lc.. of box 1)
 #pragma unroll
     for (int e = 0; e < 16; ++e) zc[e] = 0.f;
+    // rotations one tile ahead, as in the state pass
+    uint4 tab0[kTileApply / 32], tab1[kTileApply / 32];
+    auto fetch_rot = [&](int tile, int i) {
+      const long long n = (long long)tile * kTileApply + row0 + 32 * i;
+      tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
+      if (n < p.N) {
+        tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
+        if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
+      }
+    };
+    if (ROPE) {
+      TileWalk t0(wc);
+      if (!t0.done()) {
+#pragma unroll
+        for (int i = 0; i < kTileApply / 32; ++i) fetch_rot(t0.tile(), i);
+      }
+    }
     for (TileWalk t(wc); !t.done() && ok; t.next(), ++it) {
       const int s = it % NSC;
       if (t.seg_first()) {
@@ -762,7 +799,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         if (seg > 0) ok = mbar_wait(seg_done, (seg - 1) & 1, abort_flag);
         if (!ok) break;
         const int u = t.unit();
-        build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, tr, 256);
+        build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, tr, R::RELU_THREADS + 128);
         if (ROPE) {
           const float4* zrow = reinterpret_cast<const float4*>(p.state + ((size_t)u * (D + 1) + D) * D);  // G = 1: unit = (b, h)
           const float4 a0 = __ldcg(zrow + 2 * lc), a1 = __ldcg(zrow + 2 * lc + 1);
@@ -780,34 +817,27 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         // numerator operand: rotated phi(q); denominator: plain phi(q) . z, added up over the eight lanes that
         // share a row and left in the row's zero padding (features 112..) for the epilogue
         uint8_t* sl = slots + s * SLOT;
-        uint4 tab0[kTileApply / 16], tab1[kTileApply / 16];
-#pragma unroll
-        for (int i = 0; i < kTileApply / 16; ++i) {
-          const long long n = (long long)t.tile() * kTileApply + row0 + 16 * i;
-          tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
-          if (n < p.N) {
-            tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
-            if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
-          }
-        }
+        TileWalk tn = t;
+        tn.next();
         if (!__all_sync(0xffffffffu, mbar_wait(&c_full[s], (it / NSC) & 1, abort_flag))) break;  // leave as a whole warp
         uint8_t* p0 = sl + row0 * kRowBytes + pc * 16;
 #pragma unroll
-        for (int i = 0; i < kTileApply / 16; ++i) {
+        for (int i = 0; i < kTileApply / 32; ++i) {
           float f[8];
-          uint4* c0 = reinterpret_cast<uint4*>(p0 + i * 16 * kRowBytes);
+          uint4* c0 = reinterpret_cast<uint4*>(p0 + i * 32 * kRowBytes);
           unpack_relu8(*c0, f);
           float den = 0.f;
 #pragma unroll
           for (int e = 0; e < 8; ++e) den = fmaf(f[e], zc[e], den);
           *c0 = rotate_pack8(f, tab0[i]);
-          uint4* c1 = reinterpret_cast<uint4*>(p0 + HALF + i * 16 * kRowBytes);
+          uint4* c1 = reinterpret_cast<uint4*>(p0 + HALF + i * 32 * kRowBytes);
           if (box1_live) {
             unpack_relu8(*c1, f);
 #pragma unroll
             for (int e = 0; e < 8; ++e) den = fmaf(f[e], zc[8 + e], den);
             *c1 = rotate_pack8(f, tab1[i]);
           }
+          if (!tn.done()) fetch_rot(tn.tile(), i);  // this row's rotations for the next tile
           den += __shfl_xor_sync(0xffffffffu, den, 1);
           den += __shfl_xor_sync(0xffffffffu, den, 2);
           den += __shfl_xor_sync(0xffffffffu, den, 4);
@@ -822,10 +852,10 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       fence_proxy_async_smem();
       mbar_arrive(&c_ready[s]);
     }
-  } else if (warp < kStoreWarp) {
+  } else if (warp < R::STORE_WARP) {
     // ------------------------------------------------------------ epilogue: divide, round, stage the O tile
     const int wq = warp & 3;
-    const int te = threadIdx.x - kEpiThread0;
+    const int te = threadIdx.x - R::EPI_THREAD0;
     const int r = wq * 32 + lane;  // accumulator lane = token row of the tile
     uint32_t it = 0;
     for (TileWalk t(wc); !t.done(); t.next(), ++it) {
@@ -833,7 +863,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       if (t.seg_first()) {
         // this thread has seen the last accumulator of the previous segment complete: S may be rebuilt
         const int u = t.unit();
-        build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, 128 + te, 256);
+        build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, R::RELU_THREADS + te, R::RELU_THREADS + 128);
         fence_proxy_async_smem();
         mbar_arrive(s_ready);
       }
@@ -1022,7 +1052,7 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
     attr_set = true;
   }
   void* args[] = {&mk, &mv, &mq, &mo, &fp};
-  const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D, ROPE>, dim3(grid), dim3(kThreads), args,
+  const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D, ROPE>, dim3(grid), dim3(Roles<ROPE>::THREADS), args,
                                                     C::SMEM, stream);
   if (e != cudaSuccess) { cudaGetLastError(); return LINATTN_ERR_CUDA; }
   count_launches(1);
