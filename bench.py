@@ -380,6 +380,23 @@ def extras(torch, la, synth, dev, peak):
                        "algorithmic_gbs": by / (ms * 1e-3) / 1e9, "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak,
                        "l2": "one input set of %.0f MB (> 126 MB L2)" % (by / 1e6)}
         del q, k, v, o, ws
+    # Eq. 2 with its rotary factors on the 480p layer (3D table over the 21 x 30 x 52 latent grid)
+    w = synth.P480
+    q, k, v = (torch.from_numpy(x.view("int16")).to(dev).view(torch.bfloat16) for x in synth.qkv(w))
+    cos, sin = synth.rope_table(21, 30, 52, w.d)
+    table = la.rope_pack(torch.from_numpy(cos).to(dev), torch.from_numpy(sin).to(dev))
+    outs = [torch.empty_like(q) for _ in range(2)]
+    ins = [(q, k, v), (q.flip(1).contiguous(), k.flip(1).contiguous(), v.flip(1).contiguous())]
+    wsr = la.new_rope_workspace(q)
+    for i in range(3):
+        la.linattn_forward_rope(*ins[i & 1], table, w.eps, out=outs[i & 1], workspace=wsr)
+    n = 20
+    ms = time_loop(torch, lambda i: la.linattn_forward_rope(*ins[i & 1], table, w.eps, out=outs[i & 1], workspace=wsr), n) / n
+    by = w.B * w.N * w.H * 8 * w.d
+    res[w.name + "_rope"] = {"H": w.H, "d": w.d, "ms": ms, "tokens_heads_per_s": w.B * w.N * w.H / (ms * 1e-3),
+                             "algorithmic_gbs": by / (ms * 1e-3) / 1e9, "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak,
+                             "note": "q,k,v,o bytes only; the 7.3 MB fp16 rotation table is re-read from L2 by every head",
+                             "l2": "two rotating input sets of 587 MB each"}
     return res
 
 

@@ -18,7 +18,7 @@ import os
 
 __all__ = [
     "LinAttnError", "library_path", "load_library", "state_bytes", "workspace_bytes", "new_workspace",
-    "linattn_forward", "linattn_forward_rope", "rope_pack", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
+    "linattn_forward", "linattn_forward_rope", "rope_pack", "new_rope_workspace", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
 ]
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -195,6 +195,19 @@ def rope_pack(rope_cos, rope_sin):
     return table
 
 
+def new_rope_workspace(like):
+    """Allocate (with torch) and initialise a workspace for ``linattn_forward_rope`` on tensors shaped like `like`."""
+    torch = _torch()
+    lib = load_library()
+    B, N, H, d = like.shape
+    nb = ctypes.c_size_t()
+    _check(lib.linattn_rope_workspace_bytes(ctypes.byref(_Desc(B, H, d, _dtype_code(like), 0, 0, 0)), N, ctypes.byref(nb)),
+           "linattn_rope_workspace_bytes")
+    ws = torch.empty(nb.value, dtype=torch.uint8, device=like.device)
+    _check(lib.linattn_workspace_init(_ptr(ws), nb.value, _stream(like)), "linattn_workspace_init")
+    return ws
+
+
 def linattn_forward_rope(q, k, v, rope_table, eps: float = 1e-6, out=None, workspace=None):
     """Eq. 2 with its rotary factors (rotation after the ReLU, numerator only).  rope_table: the float16
     [N, d//2, 2] (cos, sin) table of ``rope_pack``: the rotation of feature pair (2p, 2p+1) of token n."""
@@ -207,10 +220,7 @@ def linattn_forward_rope(q, k, v, rope_table, eps: float = 1e-6, out=None, works
             not rope_table.is_contiguous() or rope_table.device != q.device:
         raise ValueError("rope_table must be a contiguous float16 [N, d//2, 2] tensor on the device of q")
     if workspace is None:
-        nb = ctypes.c_size_t()
-        _check(lib.linattn_rope_workspace_bytes(ctypes.byref(desc), N, ctypes.byref(nb)), "linattn_rope_workspace_bytes")
-        workspace = torch.empty(nb.value, dtype=torch.uint8, device=q.device)
-        _check(lib.linattn_workspace_init(_ptr(workspace), nb.value, _stream(q)), "linattn_workspace_init")
+        workspace = new_rope_workspace(q)
     _check(lib.linattn_forward_rope(ctypes.byref(desc), N, _ptr(q), _ptr(k), _ptr(v), _ptr(o), eps, _ptr(rope_table),
                                     _ptr(workspace), workspace.numel(), _stream(q)), "linattn_forward_rope")
     return o
