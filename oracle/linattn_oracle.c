@@ -27,6 +27,11 @@
  *   the cache is the running pair (sum S, sum phi(K)^T); a step adds the
  *   block's own (S_blk, z_blk) and then applies the block's queries to it.
  *
+ *   Eq. 2 with its rotary factors (right-hand form): RoPE after the ReLU in the
+ *   numerator only, plain denominator; linear and quadratic forms (see the
+ *   functions oracle_rope_*).  The paper fixes neither how features are paired
+ *   nor the angles: pairs are adjacent features and the rotations are inputs.
+ *
  * Readings taken where the paper is silent (each is listed in the design doc):
  *   - eps is added once to the denominator after the dot product;
  *   - a query whose phi(q).z is zero yields 0/(0+eps) = 0, never NaN;
