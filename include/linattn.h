@@ -211,6 +211,14 @@ LINATTN_API int blocklin_cache_reset(blocklin_cache* cache, void* stream);
 LINATTN_API int blocklin_step(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
                   void* o_blk, void* stream);
 
+/* blocklin_step with the rotary factors of Eq. 2 (rotation after the ReLU, numerator only): the cache then
+ * holds (sum of RoPE(phi(k))^T v, sum of phi(k)).  rope_table_blk: the packed (cos, sin) fp16 rows of this block's
+ * T_b tokens ([T_b][d/2], see linattn_forward_rope); positions simply continue from block to block, so it is
+ * usually a pointer into one table of the whole stream.  A stream uses either this call or blocklin_step for
+ * all of its blocks.  q_blk and o_blk are required. */
+LINATTN_API int blocklin_step_rope(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk,
+                                   const void* v_blk, void* o_blk, const void* rope_table_blk, void* stream);
+
 /* The denoising steps of Algorithm 1 ("x0 <- G(x; t_j, KV)" for t_j > 0): the block's queries see the
  * cache plus the block's own (S_blk, z_blk), exactly as in blocklin_step, but the cache is only read:
  * nothing is committed, blocks_seen does not change.  The clean block is committed afterwards with

@@ -52,7 +52,8 @@ def _bind(path: str):
     lib.oracle_block_step.argtypes = [sp, vp, vp, vp, f64, dp, dp, dp]
     lib.oracle_block_masked.argtypes = [sp, vp, vp, vp, f64, i64, dp]
     lib.oracle_rope_forward.argtypes = [sp, vp, vp, vp, dp, dp, f64, dp]
-    lib.oracle_rope_quadratic.argtypes = [sp, vp, vp, vp, dp, dp, f64, dp]
+    lib.oracle_rope_quadratic.argtypes = [sp, vp, vp, vp, dp, dp, f64, i64, dp]
+    lib.oracle_rope_block_masked.argtypes = [sp, vp, vp, vp, dp, dp, f64, i64, dp]
     lib.oracle_cache_bytes.argtypes = [i64, i64, i64]
     lib.oracle_cache_bytes.restype = i64
     return lib
@@ -116,16 +117,22 @@ class Oracle:
         self._lib.oracle_block_masked(ctypes.byref(s), q.ctypes.data, k.ctypes.data, v.ctypes.data, eps, T_b, self._dp(o))
         return o
 
-    def rope_forward(self, q, k, v, cos, sin, eps, quadratic: bool = False):
+    def rope_forward(self, q, k, v, cos, sin, eps, quadratic: bool = False, T_b: int = 0):
         """Eq. 2 with rotary factors in the numerator only.  cos, sin: [N, d//2] (any float dtype; widened
-        exactly to fp64), the rotation of feature pair (2p, 2p+1) of token n."""
+        exactly to fp64), the rotation of feature pair (2p, 2p+1) of token n.  T_b > 0: block-causal
+        (quadratic: masked brute force; else block by block with the running cache)."""
         s = self._shape(q, k, v)
         cs = np.ascontiguousarray(cos, dtype=np.float64)
         sn = np.ascontiguousarray(sin, dtype=np.float64)
         assert cs.shape == sn.shape == (s.N, s.d // 2)
         o = np.empty((s.B, s.N, s.H, s.d))
-        fn = self._lib.oracle_rope_quadratic if quadratic else self._lib.oracle_rope_forward
-        fn(ctypes.byref(s), q.ctypes.data, k.ctypes.data, v.ctypes.data, self._dp(cs), self._dp(sn), eps, self._dp(o))
+        args = (ctypes.byref(s), q.ctypes.data, k.ctypes.data, v.ctypes.data, self._dp(cs), self._dp(sn), eps)
+        if quadratic:
+            self._lib.oracle_rope_quadratic(*args, T_b, self._dp(o))
+        elif T_b > 0:
+            self._lib.oracle_rope_block_masked(*args, T_b, self._dp(o))
+        else:
+            self._lib.oracle_rope_forward(*args, self._dp(o))
         return o
 
     def new_cache(self, B, H, d):

@@ -274,9 +274,10 @@ void oracle_rope_forward(const oracle_shape* s, const void* q, const void* k, co
 }
 
 /* Quadratic form of the same: w_num[n][m] = RoPE_n(phi(q_n)) . RoPE_m(phi(k_m)), w_den[n][m] = phi(q_n) . phi(k_m),
- * o_n = sum_m w_num[n][m] v_m / (sum_m w_den[n][m] + eps).  O(N^2 d): tiny inputs only. */
+ * o_n = sum_m w_num[n][m] v_m / (sum_m w_den[n][m] + eps), over the tokens m that n may see (all of them, or
+ * with T_b > 0 those of its own and earlier blocks).  O(N^2 d): tiny inputs only. */
 void oracle_rope_quadratic(const oracle_shape* s, const void* q, const void* k, const void* v, const double* cs,
-                           const double* sn, double eps, double* o) {
+                           const double* sn, double eps, int64_t T_b, double* o) {
   const int64_t d = s->d, BH = s->B * s->H;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int64_t u = 0; u < BH; ++u) {
@@ -289,6 +290,7 @@ void oracle_rope_quadratic(const oracle_shape* s, const void* q, const void* k, 
       double wden = 0.0;
       for (int64_t j = 0; j < d; ++j) o_row[j] = 0.0;
       for (int64_t m = 0; m < s->N; ++m) {
+        if (T_b > 0 && (m / T_b) > (n / T_b)) continue; /* later block: not visible (T_b <= 0: no mask) */
         const int64_t kb = at(s, b, m, h);
         rope_features(s, k, kb, cs, sn, m, kp, kr);
         double wn = 0.0;
@@ -299,6 +301,47 @@ void oracle_rope_quadratic(const oracle_shape* s, const void* q, const void* k, 
       for (int64_t j = 0; j < d; ++j) o_row[j] /= wden;
     }
     free(buf);
+  }
+}
+
+/* Block-causal form with rotary factors, block by block with the cache (Eq. 3 applied to Eq. 2's right-hand
+ * form): the cache holds (sum of RoPE(phi(k))^T v, sum of phi(k)); each block is added, then its queries are
+ * applied (rotated for the numerator, plain for the denominator).  Token n of the sequence uses row n of the
+ * tables.  o: [B,N,H,d] dense fp64. */
+void oracle_rope_block_masked(const oracle_shape* s, const void* q, const void* k, const void* v, const double* cs,
+                              const double* sn, double eps, int64_t T_b, double* o) {
+  const int64_t d = s->d, BH = s->B * s->H;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t u = 0; u < BH; ++u) {
+    const int64_t b = u / s->H, h = u % s->H;
+    double* S = (double*)calloc((size_t)(d * d + 3 * d), sizeof(double));
+    double* z = S + d * d;
+    double* plain = z + d;
+    double* rot = plain + d;
+    for (int64_t n0 = 0; n0 < s->N; n0 += T_b) {
+      const int64_t n1 = n0 + T_b < s->N ? n0 + T_b : s->N;
+      for (int64_t n = n0; n < n1; ++n) { /* commit the block ... */
+        const int64_t base = at(s, b, n, h);
+        rope_features(s, k, base, cs, sn, n, plain, rot);
+        for (int64_t i = 0; i < d; ++i) {
+          z[i] += plain[i];
+          for (int64_t j = 0; j < d; ++j) S[i * d + j] += rot[i] * load_elem(v, s->dtype, base + j);
+        }
+      }
+      for (int64_t n = n0; n < n1; ++n) { /* ... then read it */
+        double* o_row = o + ((b * s->N + n) * s->H + h) * d;
+        rope_features(s, q, at(s, b, n, h), cs, sn, n, plain, rot);
+        double den = 0.0;
+        for (int64_t j = 0; j < d; ++j) o_row[j] = 0.0;
+        for (int64_t i = 0; i < d; ++i) {
+          den += plain[i] * z[i];
+          for (int64_t j = 0; j < d; ++j) o_row[j] += rot[i] * S[i * d + j];
+        }
+        den += eps;
+        for (int64_t j = 0; j < d; ++j) o_row[j] /= den;
+      }
+    }
+    free(S);
   }
 }
 

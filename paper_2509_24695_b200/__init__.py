@@ -84,6 +84,7 @@ def load_library(path: str | None = None):
         "blocklin_cache_reset": ([vp, vp], ctypes.c_int),
         "blocklin_step": ([vp, i64, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_peek": ([vp, i64, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_step_rope": ([vp, i64, vp, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_prefill": ([vp, i64, i64, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_cache_info": ([vp, ctypes.POINTER(i64), ctypes.POINTER(i64), szp], ctypes.c_int),
         "blocklin_cache_destroy": ([vp], ctypes.c_int),
@@ -363,6 +364,21 @@ class BlockLinCache:
         self._check_layout(k)
         _check(self._lib.blocklin_step(self._handle, k.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o), _stream(k)),
                "blocklin_step")
+        return o
+
+    def step_rope(self, q, k, v, rope_table_blk, out=None):
+        """``step`` with rotary factors; rope_table_blk: float16 [T_b, d//2, 2] rows of the block's tokens
+        (a contiguous slice of the stream's ``rope_pack`` table)."""
+        torch = _torch()
+        o = torch.empty_like(q) if out is None else out
+        _desc_of(q, k, v, o)
+        self._check_layout(k)
+        T_b, d = k.shape[1], k.shape[3]
+        if tuple(rope_table_blk.shape) != (T_b, d // 2, 2) or rope_table_blk.dtype != torch.float16 or \
+                not rope_table_blk.is_contiguous():
+            raise ValueError("rope_table_blk must be a contiguous float16 [T_b, d//2, 2] tensor")
+        _check(self._lib.blocklin_step_rope(self._handle, T_b, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(rope_table_blk),
+                                            _stream(k)), "blocklin_step_rope")
         return o
 
     def peek(self, q, k, v, out=None):

@@ -99,13 +99,13 @@ size_t rope_workspace_need(const Problem& p) { return round256(rope_state_offset
 
 // Eq. 2 with its rotary factors: state from the rotated keys (z from the plain ones), apply with the rotated
 // queries (denominator from the plain ones).
-int run_rope(const Problem& p, const void* q, const void* k, const void* v, void* o, float* state, float eps,
-             const __half2* rope, void* workspace, cudaStream_t stream) {
+int run_rope(const Problem& p, const void* q, const void* k, const void* v, void* o, float* state, bool accumulate,
+             float eps, const __half2* rope, void* workspace, cudaStream_t stream) {
   if (umma_rope_supported(p)) {  // one launch on the tensor cores
-    UmmaCall c{k, v, q, o, state, nullptr, false, eps, rope};
+    UmmaCall c{k, v, q, o, state, nullptr, accumulate, eps, rope};
     return umma_run(p, c, workspace, stream);
   }
-  int st = cuda_status(fma_state(p, k, v, state, false, partials_of(workspace), stream, rope));
+  int st = cuda_status(fma_state(p, k, v, state, accumulate, partials_of(workspace), stream, rope));
   if (st != LINATTN_OK) return st;
   return cuda_status(fma_apply(p, q, state, o, eps, stream, rope));
 }
@@ -334,7 +334,7 @@ int linattn_forward_rope(const linattn_desc* desc, int64_t N, const void* q, con
   if (workspace_bytes < rope_workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
   if (N == 0) return LINATTN_OK;
   float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + rope_state_offset(p));
-  return run_rope(p, q, k, v, o, state, eps, static_cast<const __half2*>(rope_table), workspace, (cudaStream_t)stream);
+  return run_rope(p, q, k, v, o, state, false, eps, static_cast<const __half2*>(rope_table), workspace, (cudaStream_t)stream);
 }
 
 uint64_t linattn_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
@@ -419,6 +419,7 @@ int blocklin_cache_bytes(const linattn_desc* desc, int64_t max_T_b, size_t* stat
   if (!state_bytes || !workspace_bytes) return LINATTN_ERR_INVALID_ARG;
   *state_bytes = sizeof(float) * (size_t)p.state_elems() * p.units();
   *workspace_bytes = workspace_need(p);
+  if ((p.d & 1) == 0 && rope_workspace_need(p) > *workspace_bytes) *workspace_bytes = rope_workspace_need(p);  // blocklin_step_rope
   return LINATTN_OK;
 }
 
@@ -470,6 +471,27 @@ int blocklin_step(blocklin_cache* cache, int64_t T_b, const void* q_blk, const v
   int st = resolve(&cache->desc, T_b, &p);
   if (st != LINATTN_OK) return st;
   return step_impl(cache, p, q_blk, k_blk, v_blk, o_blk, (cudaStream_t)stream);
+}
+
+int blocklin_step_rope(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
+                       void* o_blk, const void* rope_table_blk, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  Problem p;
+  int st = resolve(&cache->desc, T_b, &p);
+  if (st != LINATTN_OK) return st;
+  if (p.d & 1) return LINATTN_ERR_UNSUPPORTED;
+  if (p.N > 0 && (!q_blk || !k_blk || !v_blk || !o_blk || !rope_table_blk)) return LINATTN_ERR_INVALID_ARG;
+  if (o_blk && (o_blk == q_blk || o_blk == k_blk || o_blk == v_blk)) return LINATTN_ERR_INVALID_ARG;
+  if ((st = check_alignment(p, q_blk, k_blk, v_blk, o_blk)) != LINATTN_OK) return st;
+  if (!aligned16(rope_table_blk)) return LINATTN_ERR_BAD_ALIGNMENT;
+  if (cache->workspace_bytes < rope_workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  if (p.N == 0) return LINATTN_OK;
+  st = run_rope(p, q_blk, k_blk, v_blk, o_blk, cache->state, true, cache->eps, static_cast<const __half2*>(rope_table_blk),
+                cache->workspace, (cudaStream_t)stream);
+  if (st != LINATTN_OK) return st;
+  cache->blocks_seen += 1;
+  cache->tokens_seen += p.N;
+  return LINATTN_OK;
 }
 
 int blocklin_peek(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,

@@ -73,3 +73,34 @@ def test_rope_errors(la):
     with pytest.raises(la.LinAttnError) as e:
         la.linattn_forward_rope(x, x.clone(), x.clone(), t, EPS)
     assert e.value.status == -2   # odd head dim: features cannot be paired
+
+
+@pytest.mark.parametrize("case", [("bf16", 3, 112, (7, 6, 10), 60), ("f32", 2, 112, (4, 5, 5), 25), ("bf16", 2, 64, (6, 4, 8), 64),
+                                  ("bf16", 2, 112, (3, 1, 150), 150)],
+                         ids=lambda c: "%s_H%d_d%d_Tb%d" % (c[0], c[1], c[2], c[4]))
+def test_rope_block_steps_match_the_block_causal_oracle(la, orc, case):
+    """Cached block-by-block generation with rotary factors against the oracle's block-causal form; the last
+    block also equals the tail of the bidirectional rotary forward, and the cache size stays constant."""
+    import torch
+
+    dtype, H, d, (T, Hh, Ww), T_b = case
+    B, N = 1, T * Hh * Ww
+    q, k, v = gen(B, N, H, d, 5200 + N + d, dtype)
+    cos, sin = synth.rope_table(T, Hh, Ww, d)
+    table = la.rope_pack(to_dev(cos), to_dev(sin))
+    packed = table.cpu().numpy().astype(np.float64)
+    ref = orc.rope_forward(q, k, v, packed[..., 0], packed[..., 1], EPS, T_b=T_b)
+    check = assert_parity_bf16 if dtype == "bf16" else assert_parity_f32
+    cache = la.BlockLinCache(B, H, d, torch.bfloat16 if dtype == "bf16" else torch.float32, "cuda", max_T_b=T_b, eps=EPS)
+    bytes0 = cache.info()["state_bytes"]
+    outs = []
+    for n0 in range(0, N, T_b):
+        sl = slice(n0, min(n0 + T_b, N))
+        blk = [to_dev(np.ascontiguousarray(x[:, sl])) for x in (q, k, v)]
+        outs.append(cache.step_rope(*blk, table[sl].contiguous()))
+        assert cache.info()["state_bytes"] == bytes0 == B * H * (d * d + d) * 4
+    stepped = torch.cat(outs, dim=1)
+    check(to_f64(stepped), ref, f"rope steps {case}")
+    full = la.linattn_forward_rope(to_dev(q), to_dev(k), to_dev(v), table, EPS)
+    last = (N - 1) // T_b * T_b
+    check(to_f64(stepped[:, last:]), to_f64(full[:, last:]).copy(), "last block vs bidirectional rotary forward")

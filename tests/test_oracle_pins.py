@@ -325,6 +325,18 @@ def pin_rope_linear_equals_quadratic_and_shift(o):
         ones = np.ones_like(v)
         den_ratio = o.rope_forward(q, k, ones, cs, sn, EPS)          # = sum_m w_num / (sum_m w_den + eps), same in every column
         assert np.allclose(den_ratio, den_ratio[..., :1], rtol=1e-12, atol=1e-13)
+    # block-causal: cached block-by-block == masked brute force; one block == bidirectional; last block sees all
+    q, k, v = _qkv(2, 14, 2, 6, 91)
+    cs, sn, _ = _angles(14, 3, 92)
+    for T_b in (2, 4, 5, 14, 20):
+        assert np.allclose(o.rope_forward(q, k, v, cs, sn, 1e-3, T_b=T_b),
+                           o.rope_forward(q, k, v, cs, sn, 1e-3, quadratic=True, T_b=T_b), rtol=1e-9, atol=1e-10)
+    full = o.rope_forward(q, k, v, cs, sn, EPS)
+    assert np.allclose(o.rope_forward(q, k, v, cs, sn, EPS, T_b=14), full, rtol=1e-12, atol=1e-13)
+    assert np.allclose(o.rope_forward(q, k, v, cs, sn, EPS, T_b=5)[:, 10:], full[:, 10:], rtol=1e-11, atol=1e-12)
+    # ... and a block is blind to later blocks
+    k2, v2 = k.copy(), v.copy(); k2[:, 8:] += 1.0; v2[:, 8:] -= 2.0
+    assert np.array_equal(o.rope_forward(q, k, v, cs, sn, EPS, T_b=4)[:, :8], o.rope_forward(q, k2, v2, cs, sn, EPS, T_b=4)[:, :8])
     # each head and batch entry is independent, the table is shared
     q, k, v = _qkv(2, 6, 2, 4, 89)
     cs, sn, _ = _angles(6, 2, 90)
@@ -385,6 +397,10 @@ MUTANTS = {
     "rope_den_uses_rotated_query": ("        den += plain[i] * z[i];\n", "        den += rot[i] * z[i];\n"),
     "rope_state_from_plain_keys": ("S[i * d + j] += rot[i] * load_elem(v, s->dtype, base + j);", "S[i * d + j] += plain[i] * load_elem(v, s->dtype, base + j);"),
     "rope_quadratic_den_rotated": ("wden += qp[i] * kp[i];", "wden += qr[i] * kr[i];"),
+    "rope_block_mask_off": ("if (T_b > 0 && (m / T_b) > (n / T_b)) continue; /* later block: not visible (T_b <= 0: no mask) */",
+                            "if (T_b > 0 && (m / T_b) >= (n / T_b)) continue;"),
+    "rope_block_reads_before_commit": ("      for (int64_t n = n0; n < n1; ++n) { /* commit the block ... */",
+                                       "      for (int64_t n = n0; n < n0; ++n) { /* commit the block ... */"),
     "rope_token_index": ("rope_features(s, k, base, cs, sn, n, plain, rot);", "rope_features(s, k, base, cs, sn, 0, plain, rot);"),
 }
 
