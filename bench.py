@@ -366,6 +366,20 @@ def extras(torch, la, synth, dev, peak):
                        "l2": "block set of %.0f MB cycled over 3 copies" % (step_bytes / 1e6)}
         cache.close()
         del blocks, ob
+    # the 7 context blocks of the autoregressive 480p layer in one prefill call: block by block, and all together
+    w = synth.AR480
+    q, k, v = (torch.from_numpy(x.view("int16")).to(dev).view(torch.bfloat16) for x in synth.qkv(w))
+    o = torch.empty_like(q)
+    for name, nb in (("block_by_block", 0), ("all_blocks_together", w.n_blocks)):
+        cache = la.BlockLinCache(w.B, w.H, w.d, torch.bfloat16, dev, max_T_b=w.T_b, eps=w.eps, prefill_blocks=nb)
+        for _ in range(3):
+            cache.prefill(q, k, v, w.n_blocks, out=o)
+        n = 20
+        ms = time_loop(torch, lambda i: cache.prefill(q, k, v, w.n_blocks, out=o), n) / n
+        res.setdefault(w.name + "_prefill", {"blocks": w.n_blocks, "tokens": w.N,
+                                             "l2": "one 257 MB input set (> 126 MB L2)"})[name + "_us"] = ms * 1e3
+        cache.close()
+    del q, k, v, o
     # the 720p bidirectional layer and its head-dim sweep at (about) the same width
     for w in (synth.P720, synth.p720_sweep(32), synth.p720_sweep(64), synth.p720_sweep(128)):
         q, k, v = (torch.from_numpy(x.view("int16")).to(dev).view(torch.bfloat16) for x in synth.qkv(w))

@@ -86,6 +86,7 @@ def load_library(path: str | None = None):
         "blocklin_peek": ([vp, i64, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_step_rope": ([vp, i64, vp, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_prefill": ([vp, i64, i64, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_prefill_workspace_bytes": ([dp, i64, i64, szp], ctypes.c_int),
         "blocklin_cache_info": ([vp, ctypes.POINTER(i64), ctypes.POINTER(i64), szp], ctypes.c_int),
         "blocklin_cache_destroy": ([vp], ctypes.c_int),
     }
@@ -330,7 +331,7 @@ class BlockLinCache:
     """
 
     def __init__(self, B: int, H: int, d: int, dtype, device, max_T_b: int, eps: float = 1e-6,
-                 strides: tuple[int, int, int] = (0, 0, 0)):
+                 strides: tuple[int, int, int] = (0, 0, 0), prefill_blocks: int = 0):
         torch = _torch()
         self._lib = load_library()
         code = LINATTN_BF16 if dtype == torch.bfloat16 else LINATTN_F32 if dtype == torch.float32 else None
@@ -342,11 +343,17 @@ class BlockLinCache:
                "blocklin_cache_bytes")
         self.state = torch.empty((B, H, d + 1, d), dtype=torch.float32, device=device)
         assert self.state.numel() * 4 == sb.value
-        self.workspace = torch.empty(wb.value, dtype=torch.uint8, device=device)
+        nbytes = wb.value
+        if prefill_blocks > 1:  # room for prefill() to process that many blocks of max_T_b tokens together
+            pb = ctypes.c_size_t()
+            _check(self._lib.blocklin_prefill_workspace_bytes(ctypes.byref(self._desc), prefill_blocks, max_T_b,
+                                                              ctypes.byref(pb)), "blocklin_prefill_workspace_bytes")
+            nbytes = max(nbytes, pb.value)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
         self.max_T_b = max_T_b
         self._handle = ctypes.c_void_p()
         _check(self._lib.blocklin_cache_init(ctypes.byref(self._handle), ctypes.byref(self._desc), eps,
-                                             _ptr(self.state), sb.value, _ptr(self.workspace), wb.value,
+                                             _ptr(self.state), sb.value, _ptr(self.workspace), nbytes,
                                              _stream(self.state)), "blocklin_cache_init")
 
     def reset(self):

@@ -523,6 +523,34 @@ int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const
   Problem p;
   int st = resolve(&cache->desc, n_blocks * T_b, &p);
   if (st != LINATTN_OK) return st;
+  if ((st = check_alignment(p, q, k, v, o)) != LINATTN_OK) return st;
+  if (o && (o == q || o == k || o == v)) return LINATTN_ERR_INVALID_ARG;
+  // All blocks at once: with the blocks of every batch entry viewed as batch entries of their own (possible when
+  // the batch stride is that of a dense [B, n_blocks*T_b, ...] tensor), ONE state pass gives every block's own
+  // state, a prefix sum over the blocks turns them into the cache after each block (Eq. 3), and ONE apply pass
+  // reads block m's queries against prefix m.  Taken when the cache's workspace is large enough for it
+  // (blocklin_prefill_workspace_bytes); otherwise the blocks are stepped one by one.
+  Problem pv = p;
+  pv.B = p.B * (int)n_blocks;
+  pv.N = T_b;
+  pv.sb = T_b * p.sn;
+  const bool batch_dense = p.B == 1 || p.sb == n_blocks * T_b * p.sn;
+  if (n_blocks > 1 && batch_dense && (long long)pv.B * pv.H <= 65535 && (p.state_elems() * p.H) % 4 == 0 &&
+      cache->workspace_bytes >= workspace_need(pv)) {
+    cudaStream_t s = (cudaStream_t)stream;
+    float* blk = reinterpret_cast<float*>(static_cast<char*>(cache->workspace) + state_slot_offset(pv));
+    st = run_passes(pv, k, v, nullptr, nullptr, blk, false, 0.f, cache->workspace, s);
+    if (st != LINATTN_OK) return st;
+    if (prefix_states(blk, cache->state, p.B, (int)n_blocks, (long long)p.H * p.state_elems(), s) != cudaSuccess)
+      return LINATTN_ERR_CUDA;
+    if (q) {
+      st = run_passes(pv, nullptr, nullptr, q, o, blk, false, cache->eps, cache->workspace, s);
+      if (st != LINATTN_OK) return st;
+    }
+    cache->blocks_seen += n_blocks;
+    cache->tokens_seen += n_blocks * T_b;
+    return LINATTN_OK;
+  }
   p.N = T_b;
   const size_t esz = cache->desc.dtype == LINATTN_BF16 ? 2 : 4;
   for (int64_t i = 0; i < n_blocks && st == LINATTN_OK; ++i) {
@@ -532,6 +560,19 @@ int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const
                    (cudaStream_t)stream);
   }
   return st;
+}
+
+int blocklin_prefill_workspace_bytes(const linattn_desc* desc, int64_t n_blocks, int64_t T_b, size_t* workspace_bytes) {
+  Problem p;
+  if (!workspace_bytes || n_blocks < 1) return LINATTN_ERR_INVALID_ARG;
+  int st = resolve(desc, T_b, &p);
+  if (st != LINATTN_OK) return st;
+  Problem pv = p;
+  if ((long long)p.B * n_blocks * p.H > 65535) return LINATTN_ERR_UNSUPPORTED;
+  pv.B = p.B * (int)n_blocks;
+  const size_t steps = workspace_need(p), all = workspace_need(pv);
+  *workspace_bytes = all > steps ? all : steps;
+  return LINATTN_OK;
 }
 
 int blocklin_cache_info(const blocklin_cache* cache, int64_t* blocks_seen, int64_t* tokens_seen,

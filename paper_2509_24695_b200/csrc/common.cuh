@@ -49,6 +49,8 @@ cudaError_t fma_state(const Problem& p, const void* k, const void* v, float* sta
                       float* partials, cudaStream_t stream, const __half2* rope = nullptr);
 cudaError_t fma_apply(const Problem& p, const void* q, const float* state, void* o, float eps, cudaStream_t stream,
                       const __half2* rope = nullptr);
+// blk: [B][M][H][(d+1)*d] per-block states -> running states after each block (on top of cache [B][H][..]), cache := last.
+cudaError_t prefix_states(float* blk, float* cache, int B, int M, long long floats_per_batch, cudaStream_t stream);
 cudaError_t rope_pack(const float* cs, const float* sn, long long count, __half2* out, cudaStream_t stream);
 
 // ---- tensor-core (tcgen05 + TMA) kernel, bf16, d in {32 (heads contiguous), 64, 112, 128} ----

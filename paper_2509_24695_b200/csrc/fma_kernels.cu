@@ -272,7 +272,31 @@ __global__ void rope_pack_kernel(const float* __restrict__ cs, const float* __re
   if (i < count) out[i] = __floats2half2_rn(cs[i], sn[i]);
 }
 
+// Inclusive prefix over the blocks of a prefill: blk[b][m] := cache[b] + blk[b][0] + ... + blk[b][m] (added in
+// that order), cache[b] := blk[b][M-1].  One thread per float4 of a (batch, head) state.
+__global__ void prefix_states_kernel(float4* __restrict__ blk, float4* __restrict__ cache, int M, long long per_batch4) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= per_batch4) return;
+  const int b = blockIdx.y;
+  float4 run = cache[b * per_batch4 + e];
+  for (int m = 0; m < M; ++m) {
+    float4* x = blk + ((long long)b * M + m) * per_batch4 + e;
+    const float4 a = *x;
+    run.x += a.x; run.y += a.y; run.z += a.z; run.w += a.w;
+    *x = run;
+  }
+  cache[b * per_batch4 + e] = run;
+}
+
 }  // namespace
+
+cudaError_t prefix_states(float* blk, float* cache, int B, int M, long long floats_per_batch, cudaStream_t stream) {
+  const long long n4 = floats_per_batch / 4;
+  dim3 grid((unsigned)((n4 + 255) / 256), (unsigned)B);
+  prefix_states_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<float4*>(blk), reinterpret_cast<float4*>(cache), M, n4);
+  count_launches(1);
+  return cudaGetLastError();
+}
 
 cudaError_t rope_pack(const float* cs, const float* sn, long long count, __half2* out, cudaStream_t stream) {
   if (count == 0) return cudaSuccess;

@@ -56,6 +56,7 @@ def test_steps_equal_block_masked_oracle(la, orc, case, dtype):
     check = assert_parity_bf16 if dtype == "bf16" else assert_parity_f32
 
     cache = la.BlockLinCache(B, H, d, tdtype(dtype), "cuda", max_T_b=T_b, eps=EPS)
+    cache_ws_bytes = cache.workspace.numel()
     bytes0 = cache.info()["state_bytes"]
     assert bytes0 == B * H * (d * d + d) * 4 == cache.state.numel() * 4
     outs = []
@@ -83,6 +84,25 @@ def test_steps_equal_block_masked_oracle(la, orc, case, dtype):
     assert torch.equal(cache.state, final_state)
     assert cache.info()["blocks_seen"] == M
     cache.close()
+
+    # a cache with room for all M blocks takes them together (one state pass, a prefix over the blocks, one
+    # apply pass): same mathematics, sums associated differently, so the oracle is the reference again
+    big = la.BlockLinCache(B, H, d, tdtype(dtype), "cuda", max_T_b=T_b, eps=EPS, prefill_blocks=M)
+    assert big.workspace.numel() >= cache_ws_bytes
+    launches0 = la.kernel_launches()
+    o_all = big.prefill(to_dev(q), to_dev(k), to_dev(v), M)
+    assert la.kernel_launches() - launches0 <= 4   # state (+ its reduce), prefix, apply: not one set per block
+    check(to_f64(o_all), ref, f"prefill all blocks {case} {dtype}")
+    assert_state_close(to_f64(big.state), S, z, 1e-5, "cache after prefill of all blocks")
+    assert big.info() == {"blocks_seen": M, "tokens_seen": N, "state_bytes": bytes0}
+    # and it continues from a non-empty cache: a second prefill of the same blocks doubles the state
+    o_again = big.prefill(to_dev(q), to_dev(k), to_dev(v), M)
+    assert_state_close(to_f64(big.state), 2 * S, 2 * z, 1e-5, "cache after two prefills")
+    S1, z1 = orc.state(np.ascontiguousarray(k[:, :T_b]), np.ascontiguousarray(v[:, :T_b]))
+    first = orc.apply_rows(np.ascontiguousarray(q[:, :T_b]), S + S1, z + z1, EPS, np.arange(T_b))
+    check(to_f64(o_again[:, :T_b]), first, "first block of the second prefill")
+    assert la.workspace_status(big.workspace) == 0
+    big.close()
 
 
 def test_single_block_equals_forward(la):

@@ -85,6 +85,12 @@ def test_480p_block_causal_seven_steps(la, orc):
     assert torch.equal(o_pre, torch.cat(outs, dim=1))
     assert torch.equal(cache.state, final)
     assert la.workspace_status(cache.workspace) == 0
+    # with room for all seven blocks they are taken together (state pass, prefix over blocks, apply pass)
+    big = la.BlockLinCache(w.B, w.H, w.d, torch.bfloat16, "cuda", max_T_b=w.T_b, eps=w.eps, prefill_blocks=w.n_blocks)
+    o_all = big.prefill(to_dev(q), to_dev(k), to_dev(v), w.n_blocks)
+    assert_state_close(to_f64(big.state), S, z, 1e-5, "cache after prefill of all blocks")
+    assert_parity_bf16(to_f64(o_all), to_f64(o_pre), "prefill together vs block by block")
+    assert la.workspace_status(big.workspace) == 0
 
 
 def test_720p_stream_eighty_steps(la, orc):
