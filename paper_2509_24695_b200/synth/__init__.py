@@ -182,3 +182,43 @@ def rope_table(T: int, Hh: int, Ww: int, d: int, base: float = 10000.0):
     theta = np.concatenate(cols, axis=1)
     assert theta.shape == (T * Hh * Ww, half)
     return np.cos(theta).astype(np.float32), np.sin(theta).astype(np.float32)
+
+
+# ---- inputs of the temporal convolution of the Mix-FFN: x[B, T, HW, D] frames and per-channel taps w[3, D] ----
+
+X_ID, W_ID = 5, 6
+
+
+@dataclass(frozen=True)
+class ConvWorkload:
+    name: str
+    B: int
+    T: int        # frames (all blocks together)
+    HW: int       # positions of one frame
+    D: int        # channels (the model width)
+    seed: int
+    T_b: int = 0  # frames per block (0: bidirectional)
+
+
+# the 480p / 720p latent grids of the attention workloads (21 frames of 30x52 / 45x80 positions), width 2240;
+# block-causal: blocks of 3 frames (7 blocks of the 480p clip; a stretch of the 720p stream, batch 2)
+CONV_TINY = ConvWorkload("tconv_tiny", B=2, T=5, HW=6, D=16, seed=2001)
+CONV_P480 = ConvWorkload("tconv_480p_5s", B=1, T=21, HW=30 * 52, D=2240, seed=2002)
+CONV_P720 = ConvWorkload("tconv_720p_5s", B=1, T=21, HW=45 * 80, D=2240, seed=2003)
+CONV_AR480 = ConvWorkload("tconv_480p_block_causal", B=1, T=21, HW=30 * 52, D=2240, seed=2004, T_b=3)
+CONV_STREAM720 = ConvWorkload("tconv_720p_stream", B=2, T=3 * 8, HW=45 * 80, D=2240, seed=2005, T_b=3)
+
+
+def conv_frames(w: ConvWorkload, dtype: str = "bf16", t0: int = 0, frames: int | None = None) -> np.ndarray:
+    """Frames t0 .. t0+frames of the workload's x, N(0, 1) draws; the same bits whichever range is asked for."""
+    frames = w.T - t0 if frames is None else frames
+    a = np.empty((w.B, frames, w.HW, w.D), dtype=np.uint16 if dtype == "bf16" else np.float32)
+    per = w.HW * w.D
+    for b in range(w.B):
+        gauss((frames, w.HW, w.D), w.seed, X_ID, start=(b * w.T + t0) * per, dtype=dtype, out=a[b])
+    return a
+
+
+def conv_taps(D: int, seed: int, scale: float = 0.25) -> np.ndarray:
+    """Per-channel taps w[3, D] (float32), N(0, scale^2): a trained layer's taps are not known, any values do."""
+    return gauss((3, D), seed, W_ID, scale=scale, dtype="f32")
