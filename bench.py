@@ -380,6 +380,34 @@ def extras(torch, la, synth, dev, peak):
                                              "l2": "one 257 MB input set (> 126 MB L2)"})[name + "_us"] = ms * 1e3
         cache.close()
     del q, k, v, o
+    # temporal convolution of the Mix-FFN: the 480p / 720p layers, and block steps (3 frames) with the one-frame cache
+    for wl in (synth.CONV_P480, synth.CONV_P720):
+        x = torch.from_numpy(synth.conv_frames(wl).view("int16")).to(dev).view(torch.bfloat16)
+        taps = torch.from_numpy(synth.conv_taps(wl.D, wl.seed)).to(dev)
+        sets = [(x, torch.empty_like(x)), (x.flip(1).contiguous(), torch.empty_like(x))]
+        for i in range(3):
+            la.tconv_forward(sets[i & 1][0], taps, out=sets[i & 1][1])
+        n = 20
+        ms = time_loop(torch, lambda i: la.tconv_forward(sets[i & 1][0], taps, out=sets[i & 1][1]), n) / n
+        by = 2 * x.numel() * 2
+        res[wl.name] = {"B": wl.B, "frames": wl.T, "positions": wl.HW, "channels": wl.D, "ms": ms,
+                        "algorithmic_gbs": by / (ms * 1e-3) / 1e9, "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak,
+                        "l2": "two rotating sets of %.0f MB (x and y) each" % (by / 1e6)}
+        # block steps over the same frames: T_b = 3, blocks cycled so that every step's frames come from HBM
+        n_blk = wl.T // 3
+        cache = la.TConvCache(wl.B, wl.HW, wl.D, torch.bfloat16, dev)
+        xs, ys = sets[0]
+        for i in range(3):
+            cache.step(xs[:, 3 * i:3 * i + 3], taps, out=ys[:, 3 * i:3 * i + 3])
+        n = 4 * n_blk
+        ms = time_loop(torch, lambda i: cache.step(xs[:, 3 * (i % n_blk):3 * (i % n_blk) + 3], taps,
+                                                   out=ys[:, 3 * (i % n_blk):3 * (i % n_blk) + 3]), n) / n
+        by = (2 * 3 + 2) * wl.B * wl.HW * wl.D * 2      # 3 frames in and out, the cache frame read and written
+        res[wl.name + "_block_step"] = {"frames_per_block": 3, "step_latency_us": ms * 1e3,
+                                        "cache_bytes": cache.frame.numel() * 2,
+                                        "algorithmic_gbs": by / (ms * 1e-3) / 1e9, "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak,
+                                        "l2": "%d blocks of one %.0f MB tensor pair cycled" % (n_blk, 4 * x.numel() / 1e6)}
+        del x, sets, xs, ys, cache
     # the 720p bidirectional layer and its head-dim sweep at (about) the same width
     for w in (synth.P720, synth.p720_sweep(32), synth.p720_sweep(64), synth.p720_sweep(128)):
         q, k, v = (torch.from_numpy(x.view("int16")).to(dev).view(torch.bfloat16) for x in synth.qkv(w))

@@ -19,6 +19,7 @@ import os
 __all__ = [
     "LinAttnError", "library_path", "load_library", "state_bytes", "workspace_bytes", "new_workspace",
     "linattn_forward", "linattn_forward_rope", "rope_pack", "new_rope_workspace", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
+    "tconv_forward", "TConvCache",
 ]
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -38,6 +39,11 @@ class LinAttnError(RuntimeError):
 class _Desc(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("d", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("stride_b", ctypes.c_int64), ("stride_n", ctypes.c_int64), ("stride_h", ctypes.c_int64)]
+
+
+class _ConvDesc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("HW", ctypes.c_int32), ("D", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("stride_b", ctypes.c_int64), ("stride_b_y", ctypes.c_int64)]
 
 
 _lib = None
@@ -89,6 +95,11 @@ def load_library(path: str | None = None):
         "blocklin_prefill_workspace_bytes": ([dp, i64, i64, szp], ctypes.c_int),
         "blocklin_cache_info": ([vp, ctypes.POINTER(i64), ctypes.POINTER(i64), szp], ctypes.c_int),
         "blocklin_cache_destroy": ([vp], ctypes.c_int),
+        "tconv_cache_bytes": ([ctypes.POINTER(_ConvDesc), szp], ctypes.c_int),
+        "tconv_cache_reset": ([ctypes.POINTER(_ConvDesc), vp, vp], ctypes.c_int),
+        "tconv_forward": ([ctypes.POINTER(_ConvDesc), i64, vp, vp, vp, vp], ctypes.c_int),
+        "tconv_block_step": ([ctypes.POINTER(_ConvDesc), i64, vp, vp, vp, vp, ctypes.c_int, vp], ctypes.c_int),
+        "tconv_prefill": ([ctypes.POINTER(_ConvDesc), i64, i64, vp, vp, vp, vp, vp], ctypes.c_int),
     }
     for name, (argtypes, restype) in sig.items():
         fn = getattr(lib, name)
@@ -443,3 +454,92 @@ class BlockLinCache:
             self.close()
         except Exception:
             pass
+
+
+# ---- temporal convolution of the Mix-FFN (tconv.h) ----
+
+def _conv_desc_of(x, y=None) -> _ConvDesc:
+    """Descriptor for x[B, T, HW, D] (and y): frames, positions and channels dense, any batch stride."""
+    B, T, HW, D = x.shape if x.dim() == 4 else (0, 0, 0, 0)
+    strides = []
+    for t in (x, y):
+        if t is None:
+            strides.append(0)
+            continue
+        if t.dim() != 4 or not t.is_cuda or t.shape != x.shape or t.dtype != x.dtype or t.device != x.device:
+            raise ValueError("expected CUDA tensors [B, T, HW, D] of one shape, dtype and device")
+        if T > 0 and (t.stride(3) != 1 or t.stride(2) != D or (T > 1 and t.stride(1) != HW * D)):
+            raise ValueError("frames, positions and channels must be dense")
+        strides.append(t.stride(0) if B > 1 and T > 0 else 0)
+    return _ConvDesc(B, HW, D, _dtype_code(x), strides[0], strides[1])
+
+
+def _check_taps(w, D):
+    torch = _torch()
+    if w.dtype != torch.float32 or tuple(w.shape) != (3, D) or not w.is_contiguous() or not w.is_cuda:
+        raise ValueError("taps must be a contiguous CUDA float32 tensor [3, D]")
+
+
+def tconv_forward(x, w, out=None):
+    """Bidirectional temporal convolution with shortcut over x[B, T, HW, D]; taps w[3, D] float32."""
+    y = _torch().empty_like(x) if out is None else out
+    desc = _conv_desc_of(x, y)
+    _check_taps(w, x.shape[3])
+    _check(load_library().tconv_forward(ctypes.byref(desc), x.shape[1], _ptr(x), _ptr(w), _ptr(y), _stream(x)),
+           "tconv_forward")
+    return y
+
+
+class TConvCache:
+    """The conv cache of the block-causal Mix-FFN: the last frame of the previous block, [B, HW, D]."""
+
+    def __init__(self, B: int, HW: int, D: int, dtype, device):
+        torch = _torch()
+        self._lib = load_library()
+        self.frame = torch.empty((B, HW, D), dtype=dtype, device=device)
+        nbytes = ctypes.c_size_t()
+        _check(self._lib.tconv_cache_bytes(ctypes.byref(self._desc(0)), ctypes.byref(nbytes)), "tconv_cache_bytes")
+        assert nbytes.value == self.frame.numel() * self.frame.element_size()
+        self.reset()
+
+    def _desc(self, stride_b: int) -> _ConvDesc:
+        B, HW, D = self.frame.shape
+        return _ConvDesc(B, HW, D, _dtype_code(self.frame), stride_b, 0)
+
+    def _desc_for(self, x, y=None) -> _ConvDesc:
+        d = _conv_desc_of(x, y)
+        if (d.B, d.HW, d.D, d.dtype) != (self.frame.shape[0], self.frame.shape[1], self.frame.shape[2],
+                                         _dtype_code(self.frame)):
+            raise ValueError("block does not match the cache's (B, HW, D, dtype)")
+        return d
+
+    def reset(self):
+        _check(self._lib.tconv_cache_reset(ctypes.byref(self._desc(0)), _ptr(self.frame), _stream(self.frame)),
+               "tconv_cache_reset")
+
+    def step(self, x_blk, w, out=None, commit: bool = True):
+        """One block x_blk[B, T_b, HW, D]; commit=False only reads the cache (a denoising step)."""
+        y = _torch().empty_like(x_blk) if out is None else out
+        d = self._desc_for(x_blk, y)
+        _check_taps(w, d.D)
+        _check(self._lib.tconv_block_step(ctypes.byref(d), x_blk.shape[1], _ptr(x_blk), _ptr(w), _ptr(self.frame),
+                                          _ptr(y), int(commit), _stream(x_blk)), "tconv_block_step")
+        return y
+
+    def absorb(self, x_blk):
+        """Take a block into the cache without computing its output."""
+        d = self._desc_for(x_blk)
+        _check(self._lib.tconv_block_step(ctypes.byref(d), x_blk.shape[1], _ptr(x_blk), None, _ptr(self.frame), None, 1,
+                                          _stream(x_blk)), "tconv_block_step")
+
+    def prefill(self, x, w, n_blocks: int, out=None):
+        """n_blocks equal blocks of x[B, n_blocks*T_b, HW, D] in one launch."""
+        T = x.shape[1]
+        if n_blocks <= 0 or T % n_blocks:
+            raise ValueError("frame count must be n_blocks * T_b")
+        y = _torch().empty_like(x) if out is None else out
+        d = self._desc_for(x, y)
+        _check_taps(w, d.D)
+        _check(self._lib.tconv_prefill(ctypes.byref(d), n_blocks, T // n_blocks, _ptr(x), _ptr(w), _ptr(self.frame),
+                                       _ptr(y), _stream(x)), "tconv_prefill")
+        return y

@@ -34,7 +34,7 @@ def sources() -> list[str]:
 
 def _fingerprint() -> str:
     h = hashlib.sha256()
-    files = sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + [os.path.join(ROOT, "include", "linattn.h")]
+    files = sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + sorted(glob.glob(os.path.join(ROOT, "include", "*.h")))
     for f in files:
         h.update(f.encode())
         h.update(open(f, "rb").read())

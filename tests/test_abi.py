@@ -18,14 +18,17 @@ def lib():
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "linattn.h")).read()
-    return sorted(set(re.findall(r"LINATTN_API\s+[\w\s\*]+?\b((?:linattn|blocklin)_\w+)\s*\(", text)))
+    import glob
+
+    text = "".join(open(h).read() for h in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))))
+    return sorted(set(re.findall(r"LINATTN_API\s+[\w\s\*]+?\b((?:linattn|blocklin|tconv)_\w+)\s*\(", text)))
 
 
 def test_header_symbols_are_exported(lib):
     names = declared_symbols()
     assert {"linattn_forward", "linattn_state", "linattn_apply", "blocklin_cache_init", "blocklin_cache_reset",
-            "blocklin_step", "blocklin_prefill"} <= set(names)
+            "blocklin_step", "blocklin_prefill", "tconv_forward", "tconv_block_step", "tconv_prefill",
+            "tconv_cache_bytes", "tconv_cache_reset"} <= set(names)
     for n in names:
         assert hasattr(lib, n), f"{n} declared in linattn.h but not exported"
 
@@ -34,7 +37,8 @@ def test_header_compiles_as_plain_c(tmp_path):
     import subprocess
 
     src = tmp_path / "t.c"
-    src.write_text('#include "linattn.h"\nint main(void){ linattn_desc d; (void)d; return LINATTN_OK; }\n')
+    src.write_text('#include "linattn.h"\n#include "tconv.h"\n'
+                   'int main(void){ linattn_desc d; tconv_desc c; (void)d; (void)c; return LINATTN_OK; }\n')
     subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), "-c", str(src),
                            "-o", str(tmp_path / "t.o")])
 
@@ -79,3 +83,22 @@ def test_product_package_does_not_touch_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".c", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in text and "from oracle" not in text and "liblinattn_oracle" not in text, f
+
+
+def test_tconv_sizes_and_validation_without_gpu(lib):
+    import paper_2509_24695_b200 as la
+
+    nbytes = ctypes.c_size_t()
+    d = la._ConvDesc(2, 30 * 52, 2240, 0, 0, 0)
+    assert lib.tconv_cache_bytes(ctypes.byref(d), ctypes.byref(nbytes)) == 0
+    assert nbytes.value == 2 * 30 * 52 * 2240 * 2            # one frame per batch entry, nothing per block
+    d32 = la._ConvDesc(1, 10, 16, 1, 0, 0)
+    assert lib.tconv_cache_bytes(ctypes.byref(d32), ctypes.byref(nbytes)) == 0 and nbytes.value == 10 * 16 * 4
+    assert lib.tconv_cache_bytes(ctypes.byref(la._ConvDesc(1, 10, 12, 0, 0, 0)), ctypes.byref(nbytes)) == -2
+    assert lib.tconv_cache_bytes(ctypes.byref(la._ConvDesc(0, 10, 16, 0, 0, 0)), ctypes.byref(nbytes)) == -1
+    assert lib.tconv_cache_bytes(None, ctypes.byref(nbytes)) == -1
+    # null tensors and negative sizes are rejected before any launch
+    assert lib.tconv_forward(ctypes.byref(d), 3, None, None, None, None) == -1
+    assert lib.tconv_forward(ctypes.byref(d), -1, None, None, None, None) == -1
+    assert lib.tconv_block_step(ctypes.byref(d), 3, None, None, None, None, 1, None) == -1
+    assert lib.tconv_prefill(ctypes.byref(d), -1, 3, None, None, None, None, None) == -1
