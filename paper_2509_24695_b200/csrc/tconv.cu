@@ -5,8 +5,7 @@
 // written once; 2 * sizeof(element) bytes per element is all that has to cross HBM.  One thread owns
 // 16 bytes of a frame (8 bf16 / 4 fp32 channels of one position) and walks the frame axis with the previous,
 // current and next frame's values in registers, so x is read from memory exactly once and no shared memory or
-// cache reuse is involved; the loads of the frame after next are issued before the current frame's arithmetic,
-// which keeps three 16-byte loads per thread in flight.  Consecutive threads take consecutive 16-byte pieces
+// cache reuse is involved; the loads of three further frames are in flight while a frame is computed.  Consecutive threads take consecutive 16-byte pieces
 // (fully coalesced 512-byte warp accesses).  The cached frame is read by, and the new cache written by, the same
 // thread that owns that piece, so updating the cache in place needs no ordering between threads.
 #include <cuda_bf16.h>
@@ -18,52 +17,55 @@
 namespace linattn {
 namespace {
 
-// 16 bytes of T: kept packed in registers, widened to floats only where the arithmetic happens
+// 16 bytes of a frame as they sit in memory, and as pairs of floats for the arithmetic
 template <typename T>
-struct Vec;
+struct Piece;
 
 template <>
-struct Vec<__nv_bfloat16> {
-  static constexpr int N = 8;
-  uint4 r;
-  __device__ __forceinline__ void load(const __nv_bfloat16* p) { r = __ldcs(reinterpret_cast<const uint4*>(p)); }
-  __device__ __forceinline__ void zero() { r = make_uint4(0, 0, 0, 0); }
-  __device__ __forceinline__ void unpack(float (&f)[8]) const {
+struct Piece<__nv_bfloat16> {
+  static constexpr int PAIRS = 4;
+  using Raw = uint4;
+  static __device__ __forceinline__ Raw zero() { return make_uint4(0, 0, 0, 0); }
+  static __device__ __forceinline__ void unpack(const Raw& r, float2 (&f)[4]) {
     const unsigned u[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      f[2 * i] = __uint_as_float(u[i] << 16);
-      f[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
-    }
+    for (int i = 0; i < 4; ++i) f[i] = make_float2(__uint_as_float(u[i] << 16), __uint_as_float(u[i] & 0xffff0000u));
   }
-  __device__ __forceinline__ void pack(const float (&f)[8]) {
+  static __device__ __forceinline__ Raw pack(const float2 (&f)[4]) {   // round to nearest even
     unsigned u[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      const __nv_bfloat162 h = __floats2bfloat162_rn(f[i].x, f[i].y);
       u[i] = *reinterpret_cast<const unsigned*>(&h);
     }
-    r = make_uint4(u[0], u[1], u[2], u[3]);
-  }
-  __device__ __forceinline__ void store(__nv_bfloat16* p, bool streaming) const {
-    if (streaming) __stcs(reinterpret_cast<uint4*>(p), r);
-    else *reinterpret_cast<uint4*>(p) = r;
+    return make_uint4(u[0], u[1], u[2], u[3]);
   }
 };
 
 template <>
-struct Vec<float> {
-  static constexpr int N = 4;
-  float4 r;
-  __device__ __forceinline__ void load(const float* p) { r = __ldcs(reinterpret_cast<const float4*>(p)); }
-  __device__ __forceinline__ void zero() { r = make_float4(0.f, 0.f, 0.f, 0.f); }
-  __device__ __forceinline__ void unpack(float (&f)[4]) const { f[0] = r.x; f[1] = r.y; f[2] = r.z; f[3] = r.w; }
-  __device__ __forceinline__ void pack(const float (&f)[4]) { r = make_float4(f[0], f[1], f[2], f[3]); }
-  __device__ __forceinline__ void store(float* p, bool streaming) const {
-    if (streaming) __stcs(reinterpret_cast<float4*>(p), r);
-    else *reinterpret_cast<float4*>(p) = r;
+struct Piece<float> {
+  static constexpr int PAIRS = 2;
+  using Raw = float4;
+  static __device__ __forceinline__ Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+  static __device__ __forceinline__ void unpack(const Raw& r, float2 (&f)[2]) {
+    f[0] = make_float2(r.x, r.y);
+    f[1] = make_float2(r.z, r.w);
   }
+  static __device__ __forceinline__ Raw pack(const float2 (&f)[2]) { return make_float4(f[0].x, f[0].y, f[1].x, f[1].y); }
 };
+
+// Two fp32 fused multiply-adds in one instruction (sm_100 has a packed f32x2 FMA pipe): the kernel issues an
+// instruction on every other cycle per scheduler as it is, so halving the FMA count shows in the run time.
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  unsigned long long ra, rb, rc, rd;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rc) : "f"(c.x), "f"(c.y));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+  float2 d;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+  return d;
+}
 
 struct TconvParams {
   const void* x;
@@ -77,57 +79,67 @@ struct TconvParams {
   int D;
 };
 
+constexpr int kAhead = 3;   // frames in flight beyond the next one
+
 template <typename T>
-__global__ void __launch_bounds__(256, 4) tconv_kernel(const TconvParams p) {
-  using V = Vec<T>;
-  const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V::N;   // element within a frame
+__global__ void __launch_bounds__(256, 3) tconv_kernel(const TconvParams p) {
+  using Pc = Piece<T>;
+  using Raw = typename Pc::Raw;
+  constexpr int PAIRS = Pc::PAIRS;
+  const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * (2 * PAIRS);   // element within a frame
   if (col >= p.frame) return;
   const int b = blockIdx.y;
   const T* x = static_cast<const T*>(p.x) + b * p.sb + col;
-  T* cache_out = p.cache_out ? static_cast<T*>(p.cache_out) + b * p.frame + col : nullptr;
+  Raw* cache_out = p.cache_out ? reinterpret_cast<Raw*>(static_cast<T*>(p.cache_out) + b * p.frame + col) : nullptr;
+  auto frame_of = [&](long long t) { return __ldcs(reinterpret_cast<const Raw*>(x + t * p.frame)); };
   if (!p.y) {  // absorb only: the cache becomes the last frame
-    V last;
-    last.load(x + (p.T - 1) * p.frame);
-    if (cache_out) last.store(cache_out, false);
+    if (cache_out) *cache_out = frame_of(p.T - 1);
     return;
   }
   T* y = static_cast<T*>(p.y) + b * p.sby + col;
 
   const int c0 = (int)(col % p.D);
-  float w0[V::N], w1[V::N], w2[V::N];
+  float2 w[3][PAIRS];
 #pragma unroll
-  for (int i = 0; i < V::N; i += 4) {
-    const float4 a = __ldg(reinterpret_cast<const float4*>(p.w + c0 + i));
-    const float4 c = __ldg(reinterpret_cast<const float4*>(p.w + p.D + c0 + i));
-    const float4 d = __ldg(reinterpret_cast<const float4*>(p.w + 2 * p.D + c0 + i));
-    w0[i] = a.x; w0[i + 1] = a.y; w0[i + 2] = a.z; w0[i + 3] = a.w;
-    w1[i] = c.x; w1[i + 1] = c.y; w1[i + 2] = c.z; w1[i + 3] = c.w;
-    w2[i] = d.x; w2[i + 1] = d.y; w2[i + 2] = d.z; w2[i + 3] = d.w;
-  }
+  for (int tau = 0; tau < 3; ++tau)
+#pragma unroll
+    for (int i = 0; i < PAIRS; i += 2) {
+      const float4 a = __ldg(reinterpret_cast<const float4*>(p.w + tau * p.D + c0 + 2 * i));
+      w[tau][i] = make_float2(a.x, a.y);
+      w[tau][i + 1] = make_float2(a.z, a.w);
+    }
 
-  V prev, cur, nxt, ahead;
-  if (p.cache_in) prev.load(static_cast<const T*>(p.cache_in) + b * p.frame + col);
-  else prev.zero();
-  cur.load(x);
-  if (p.T > 1) nxt.load(x + p.frame); else nxt.zero();
+  // frames t-1, t, t+1 as floats (each frame is widened once), frames t+2 .. t+1+kAhead as loaded
+  Raw r_prev = Pc::zero(), r_cur, r_nxt = Pc::zero(), raw[kAhead];
+  if (p.cache_in) r_prev = __ldcs(reinterpret_cast<const Raw*>(static_cast<const T*>(p.cache_in) + b * p.frame + col));
+  r_cur = frame_of(0);
+  if (p.T > 1) r_nxt = frame_of(1);
+#pragma unroll
+  for (int i = 0; i < kAhead; ++i) raw[i] = 2 + i < p.T ? frame_of(2 + i) : Pc::zero();
+  float2 fp[PAIRS], fc[PAIRS], fn[PAIRS];
+  Pc::unpack(r_prev, fp); Pc::unpack(r_cur, fc); Pc::unpack(r_nxt, fn);
   long long in_block = 0;   // index of frame t within its block
   for (long long t = 0; t < p.T; ++t) {
-    if (t + 2 < p.T) ahead.load(x + (t + 2) * p.frame); else ahead.zero();
-    const bool block_end = ++in_block == p.T_b || t + 1 == p.T;
+    Raw fresh = Pc::zero();
+    if (t + 2 + kAhead < p.T) fresh = frame_of(t + 2 + kAhead);
+    const bool block_end = ++in_block == p.T_b || t + 1 == p.T;   // the same for every thread: no divergence
     if (block_end) in_block = 0;
-    float fp[V::N], fc[V::N], fn[V::N], fo[V::N];
-    prev.unpack(fp); cur.unpack(fc); nxt.unpack(fn);
+    float2 fo[PAIRS];
 #pragma unroll
-    for (int i = 0; i < V::N; ++i) {
-      const float n = block_end ? 0.f : fn[i];
-      fo[i] = fmaf(w2[i], n, fmaf(w1[i], fc[i], fmaf(w0[i], fp[i], fc[i])));
+    for (int i = 0; i < PAIRS; ++i) fo[i] = fma2(w[1][i], fc[i], fma2(w[0][i], fp[i], fc[i]));
+    if (!block_end) {   // behind a block's last frame stands the all-zero frame: nothing to add
+#pragma unroll
+      for (int i = 0; i < PAIRS; ++i) fo[i] = fma2(w[2][i], fn[i], fo[i]);
     }
-    V out;
-    out.pack(fo);
-    out.store(y + t * p.frame, true);
-    prev = cur; cur = nxt; nxt = ahead;
+    __stcs(reinterpret_cast<Raw*>(y + t * p.frame), Pc::pack(fo));
+#pragma unroll
+    for (int i = 0; i < PAIRS; ++i) { fp[i] = fc[i]; fc[i] = fn[i]; }
+    Pc::unpack(raw[0], fn);
+#pragma unroll
+    for (int i = 0; i + 1 < kAhead; ++i) raw[i] = raw[i + 1];
+    raw[kAhead - 1] = fresh;
   }
-  if (cache_out) prev.store(cache_out, false);   // prev is now the last frame
+  if (cache_out) *cache_out = Pc::pack(fp);   // fp is now the last frame; packing widened elements is exact
 }
 
 int check(const tconv_desc* d, long long T, long long* frame, long long* sb, long long* sby, size_t* esz) {
