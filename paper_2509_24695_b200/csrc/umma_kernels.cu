@@ -290,71 +290,110 @@ __device__ __forceinline__ void grid_barrier(WorkspaceCtrl* ctrl, volatile int* 
 // ---------------------------------------------------------------- reduce
 // This CTA's slice of the state: state[b][h][e] = (accumulate ? state : 0) + the partial records of
 // the head's unit, column CTAs first (ascending), then the trailing CTAs (ascending).
+//
+// The reduce sits between two grid barriers with HBM idle, so it is written for latency: a thread takes
+// up to NE elements (float4) of the slice, works out where all their records are, issues every load
+// (NE x NR independent 16-byte loads, plus the old state when accumulating) and only then adds, in the
+// fixed order.  Index arithmetic is 32-bit wherever the sizes allow: 64-bit division is a long
+// subroutine, and a handful of them per element used to cost more time than the loads.
+
+// Trailing CTA r covers the flat positions [r*tot/R, (r+1)*tot/R) (work_of); the one that holds position f is
+// the largest r with r*tot/R <= f, i.e. floor(((f+1)*R - 1) / tot): one division.
 __device__ __forceinline__ int trailing_cta_of(long long f, long long tot, int R) {
-  long long r = f * R / tot;
-  while (r + 1 < R && (r + 1) * tot / R <= f) ++r;
-  while (r > 0 && r * tot / R > f) --r;
-  return (int)r;
+  if ((tot + 1) * R < 0xffffffffLL) return (int)((((unsigned)f + 1u) * (unsigned)R - 1u) / (unsigned)tot);
+  return (int)(((f + 1) * R - 1) / tot);
 }
 
 __device__ __forceinline__ void add4(float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
 
-template <int D, bool ROPE>
-__device__ void reduce_slice(const FusedParams& p) {
+template <int D, bool ROPE, int NE, int NR>
+__device__ __forceinline__ void reduce_elements(const FusedParams& p, int first, int i1, int ncol) {
   using C = Cfg<D>;
   constexpr int E4 = (D + 1) * D / 4;  // float4 per head state
   constexpr int REC4 = C::G * E4 + (ROPE ? kZParts / 4 : 0);  // float4 per partial record
   const Sched& s = p.sa;
-  const long long tot = (long long)p.B * p.H * E4;
-  const long long i0 = (long long)blockIdx.x * tot / gridDim.x;
-  const long long i1 = (long long)(blockIdx.x + 1) * tot / gridDim.x;
-  const int ncol = s.P == 0 ? 0 : (s.P < (s.tpu + s.Lc - 1) / s.Lc ? s.P : (s.tpu + s.Lc - 1) / s.Lc);
   const long long ttot = (long long)s.U * s.m;
   float4* state4 = reinterpret_cast<float4*>(p.state);
-  for (long long idx = i0 + threadIdx.x; idx < i1; idx += blockDim.x) {
-    const int bh = (int)(idx / E4), e = (int)(idx % E4);
-    const int b = bh / p.H, h = bh % p.H;
+  const float4* src[NE];
+  int u_of[NE], r_lo[NE], nrec[NE];
+  bool live[NE], zpart[NE];
+  float4 sum[NE], v[NE][NR];
+#pragma unroll
+  for (int k = 0; k < NE; ++k) {
+    const int idx = first + k * (int)blockDim.x;
+    live[k] = idx < i1;
+    zpart[k] = false;
+    if (!live[k]) continue;
+    sum[k] = p.accumulate ? __ldcg(reinterpret_cast<const float4*>(p.state_base) + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+    const int bh = idx / E4, e = idx - bh * E4;
+    const int b = bh / p.H, h = bh - b * p.H;
     const int u = b * p.HG + h / C::G, g = h % C::G;
-    const float4* src = reinterpret_cast<const float4*>(p.partials) + (size_t)g * E4 + e;
-    float4 sum = p.accumulate ? __ldcg(reinterpret_cast<const float4*>(p.state_base) + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
-    // every record of the unit, column CTAs first, then the trailing CTAs; the loads of a batch are
-    // independent and issued together, the adds keep that fixed order
-    int r_lo = 0, ntrail = 0;
+    u_of[k] = u;
+    src[k] = reinterpret_cast<const float4*>(p.partials) + (size_t)g * E4 + e;
+    int ntrail = 0;
+    r_lo[k] = 0;
     if (s.m > 0) {
-      r_lo = trailing_cta_of((long long)u * s.m, ttot, s.R);
-      ntrail = trailing_cta_of((long long)(u + 1) * s.m - 1, ttot, s.R) - r_lo + 1;
+      r_lo[k] = trailing_cta_of((long long)u * s.m, ttot, s.R);
+      ntrail = trailing_cta_of((long long)(u + 1) * s.m - 1, ttot, s.R) - r_lo[k] + 1;
     }
-    const int nrec = ncol + ntrail;
-    if (ROPE && e >= D * D / 4) {
-      // rotary variant: z comes from the plain phi(k) sums that the four ReLU warps of every segment left
+    nrec[k] = ncol + ntrail;
+    zpart[k] = ROPE && e >= D * D / 4;
+  }
+  auto record_of = [&](int k, int kk) { return kk < ncol ? kk * s.U + u_of[k] : s.P * s.U + r_lo[k] + (kk - ncol) + u_of[k]; };
+  int nmax = 0;
+#pragma unroll
+  for (int k = 0; k < NE; ++k)
+    if (live[k] && !zpart[k] && nrec[k] > nmax) nmax = nrec[k];
+  for (int k0 = 0; k0 < nmax; k0 += NR) {
+#pragma unroll
+    for (int k = 0; k < NE; ++k)
+#pragma unroll
+      for (int r = 0; r < NR; ++r)
+        if (live[k] && !zpart[k] && k0 + r < nrec[k]) v[k][r] = __ldcg(src[k] + (size_t)record_of(k, k0 + r) * REC4);
+#pragma unroll
+    for (int k = 0; k < NE; ++k)
+#pragma unroll
+      for (int r = 0; r < NR; ++r)
+        if (live[k] && !zpart[k] && k0 + r < nrec[k]) add4(sum[k], v[k][r]);
+  }
+#pragma unroll
+  for (int k = 0; k < NE; ++k) {
+    if (!live[k]) continue;
+    const int idx = first + k * (int)blockDim.x;
+    if (ROPE && zpart[k]) {
+      // rotary variant: z comes from the plain phi(k) sums that the ReLU warps of every segment left
       // behind the record (per warp, per feature); records in their fixed order, warps 0..7 within each
+      const int e = idx % E4;
       const float4* zp = reinterpret_cast<const float4*>(p.partials) + E4 + (e - D * D / 4);
-      for (int kk = 0; kk < nrec; ++kk) {
-        const int rec = kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u;
+      for (int kk = 0; kk < nrec[k]; ++kk) {
         float4 w4[8];
 #pragma unroll
-        for (int w = 0; w < 8; ++w) w4[w] = __ldcg(zp + (size_t)rec * REC4 + w * 32);
+        for (int w = 0; w < 8; ++w) w4[w] = __ldcg(zp + (size_t)record_of(k, kk) * REC4 + w * 32);
 #pragma unroll
-        for (int w = 0; w < 8; ++w) add4(sum, w4[w]);
+        for (int w = 0; w < 8; ++w) add4(sum[k], w4[w]);
       }
-      state4[idx] = sum;
-      continue;
     }
-    for (int k0 = 0; k0 < nrec; k0 += 12) {
-      float4 v[12];
-#pragma unroll
-      for (int k = 0; k < 12; ++k) {
-        const int kk = k0 + k;
-        if (kk < nrec) {
-          const int rec = kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u;
-          v[k] = __ldcg(src + (size_t)rec * REC4);
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < 12; ++k)
-        if (k0 + k < nrec) add4(sum, v[k]);
-    }
-    state4[idx] = sum;
+    state4[idx] = sum[k];
+  }
+}
+
+template <int D, bool ROPE>
+__device__ void reduce_slice(const FusedParams& p) {
+  constexpr int E4 = (D + 1) * D / 4;
+  const Sched& s = p.sa;
+  const int tot = p.B * p.H * E4;   // < 2^31: at most 65535 units of at most 4128 float4
+  const int per = tot / (int)gridDim.x, rem = tot - per * (int)gridDim.x, me = (int)blockIdx.x;
+  const int i0 = me * per + (me < rem ? me : rem);
+  const int i1 = i0 + per + (me < rem ? 1 : 0);
+  const int ncol = s.P == 0 ? 0 : (s.P < (s.tpu + s.Lc - 1) / s.Lc ? s.P : (s.tpu + s.Lc - 1) / s.Lc);
+  // few elements per thread: more records per batch; more elements: fewer records each (about 20 loads either way;
+  // half as many in the rotary variant, whose 480 threads have 128 registers each)
+  if (i1 - i0 <= 2 * (int)blockDim.x) {
+    for (int first = i0 + (int)threadIdx.x; first < i1; first += 2 * (int)blockDim.x)
+      reduce_elements<D, ROPE, 2, ROPE ? 5 : 10>(p, first, i1, ncol);
+  } else {
+    for (int first = i0 + (int)threadIdx.x; first < i1; first += 3 * (int)blockDim.x)
+      reduce_elements<D, ROPE, 3, ROPE ? 3 : 6>(p, first, i1, ncol);
   }
 }
 
