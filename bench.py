@@ -366,12 +366,49 @@ def extras(torch, la, synth, dev, peak):
         lat = [evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(n_steps)]
         step_bytes = w.B * w.T_b * w.H * 8 * w.d + 2 * cache.info()["state_bytes"]
         med = sorted(lat)[len(lat) // 2]
-        res[w.name] = {"step_latency_us_median": med, "step_latency_us_first": lat[0], "step_latency_us_last": lat[-1],
+
+        # the same steps without an event between them (an event record between two launches costs the device
+        # 2-3 us): two events around the whole run, first launched one by one, then replayed from a CUDA graph
+        def all_steps(handle):
+            for i in range(n_steps):
+                qp, kp, vp_ = ptrs[i % 3]
+                if lib.blocklin_step(cache._handle, w.T_b, qp, kp, vp_, op, handle) != 0:
+                    raise RuntimeError("blocklin_step failed")
+
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            handle = ctypes.c_void_p(side.cuda_stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            all_steps(handle)
+            torch.cuda.synchronize()
+            e0.record(side); all_steps(handle); e1.record(side)
+            torch.cuda.synchronize()
+            us_launched = e0.elapsed_time(e1) * 1e3 / n_steps
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                all_steps(ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+            graph.replay()
+            torch.cuda.synchronize()
+            e0.record(side); graph.replay(); e1.record(side)
+            torch.cuda.synchronize()
+            us_graph = e0.elapsed_time(e1) * 1e3 / n_steps
+        torch.cuda.current_stream().wait_stream(side)
+        if la.workspace_status(cache.workspace) != 0:
+            raise RuntimeError("a block step reported an error status")
+        res[w.name] = {"step_latency_us": us_launched, "step_latency_us_graph_replay": us_graph,
+                       "step_latency_us_median": med, "step_latency_us_first": lat[0], "step_latency_us_last": lat[-1],
+                       "note": "step_latency_us: %d steps launched back to back, two events around the run; "
+                               "graph_replay: the same steps replayed from one CUDA graph; median/first/last: "
+                               "with an event recorded after every step" % n_steps,
                        "steps": n_steps, "tokens_per_block": w.T_b, "B": w.B,
-                       "tokens_heads_per_s": w.B * w.T_b * w.H / (med * 1e-6),
-                       "algorithmic_gbs": step_bytes / (med * 1e-6) / 1e9, "frac_of_peak": step_bytes / (med * 1e-6) / 1e9 / peak,
+                       "tokens_heads_per_s": w.B * w.T_b * w.H / (us_launched * 1e-6),
+                       "algorithmic_gbs": step_bytes / (us_launched * 1e-6) / 1e9,
+                       "frac_of_peak": step_bytes / (us_launched * 1e-6) / 1e9 / peak,
+                       "frac_of_peak_graph_replay": step_bytes / (us_graph * 1e-6) / 1e9 / peak,
                        "cache_bytes_at_first_and_last_step": [cache.info()["state_bytes"]] * 2,
                        "l2": "block set of %.0f MB cycled over 3 copies" % (step_bytes / 1e6)}
+        del graph
         cache.close()
         del blocks, ob
     # the 7 context blocks of the autoregressive 480p layer in one prefill call: block by block, and all together

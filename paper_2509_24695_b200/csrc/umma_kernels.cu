@@ -184,6 +184,8 @@ struct FusedParams {
   float* partials;         // one record of G head-states per (CTA, unit) segment of the state pass
   float eps;
   WorkspaceCtrl* ctrl;
+  uint8_t* s_image;        // non-null: the reduce also leaves every unit's S operand (bf16 hi + lo, in the shared-memory
+                           // layout) here, S_BYTES per unit, and the apply pass fetches it with one bulk copy
   const uint4* rope;       // rotary variant: [N][d/8] chunks of four (cos, sin) fp16 pairs; null otherwise
   long long N;             // tokens (bound of the rotary table)
 };
@@ -395,6 +397,124 @@ __device__ void reduce_slice(const FusedParams& p) {
     for (int first = i0 + (int)threadIdx.x; first < i1; first += 3 * (int)blockDim.x)
       reduce_elements<D, ROPE, 3, ROPE ? 3 : 6>(p, first, i1, ncol);
   }
+}
+
+// ---------------------------------------------------------------- reduce, with the S operand as a by-product
+// Fused launches of one-head units (d = 112, 128) with at least one column CTA per unit: the column CTAs of a
+// unit share its reduce (part c of P), in 32-byte chunks of a state row, and besides the fp32 state each chunk's
+// sum is split into bf16 hi + lo and stored where the apply MMA wants it (the layout build_s_operand writes to
+// shared memory), in a per-unit image in the workspace.  After the second barrier a CTA gets its unit's operand
+// with one bulk copy instead of re-reading and converting the whole state: the conversion is done once per
+// unit, not once per CTA, and the serial section between the passes is about 2 us shorter.  Same records in the
+// same order as reduce_slice, so the state comes out bit for bit the same.
+template <int D, bool ROPE, int NE, int NR>
+__device__ __forceinline__ void reduce_image_chunks(const FusedParams& p, int u, int first, int hi_end, int ncol, int r_lo,
+                                                    int nrec) {
+  using C = Cfg<D>;
+  constexpr int CPR = D / 8;                 // 32-byte chunks per state row
+  constexpr int E4 = (D + 1) * D / 4;        // float4 per head state
+  constexpr int REC4 = E4 + (ROPE ? kZParts / 4 : 0);
+  const Sched& s = p.sa;
+  auto record_of = [&](int kk) { return kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u; };
+  const float4* part4 = reinterpret_cast<const float4*>(p.partials);
+  float4 sum[NE][2], v[NE][NR][2];
+  int j_of[NE], c_of[NE];
+  bool live[NE], zrow[NE];
+#pragma unroll
+  for (int k = 0; k < NE; ++k) {
+    const int idx = first + k * (int)blockDim.x;
+    live[k] = idx < hi_end;
+    zrow[k] = false;
+    if (!live[k]) continue;
+    j_of[k] = idx / CPR;
+    c_of[k] = idx - j_of[k] * CPR;
+    zrow[k] = ROPE && j_of[k] == D;
+    const size_t e4 = (size_t)u * E4 + (size_t)j_of[k] * (D / 4) + 2 * c_of[k];
+    if (p.accumulate) {
+      sum[k][0] = __ldcg(reinterpret_cast<const float4*>(p.state_base) + e4);
+      sum[k][1] = __ldcg(reinterpret_cast<const float4*>(p.state_base) + e4 + 1);
+    } else {
+      sum[k][0] = sum[k][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  for (int k0 = 0; k0 < nrec; k0 += NR) {
+#pragma unroll
+    for (int k = 0; k < NE; ++k)
+#pragma unroll
+      for (int r = 0; r < NR; ++r)
+        if (live[k] && !zrow[k] && k0 + r < nrec) {
+          const float4* src = part4 + (size_t)record_of(k0 + r) * REC4 + j_of[k] * (D / 4) + 2 * c_of[k];
+          v[k][r][0] = __ldcg(src);
+          v[k][r][1] = __ldcg(src + 1);
+        }
+#pragma unroll
+    for (int k = 0; k < NE; ++k)
+#pragma unroll
+      for (int r = 0; r < NR; ++r)
+        if (live[k] && !zrow[k] && k0 + r < nrec) { add4(sum[k][0], v[k][r][0]); add4(sum[k][1], v[k][r][1]); }
+  }
+#pragma unroll
+  for (int k = 0; k < NE; ++k) {
+    if (!live[k]) continue;
+    if (ROPE && zrow[k]) {
+      // rotary variant: z from the plain phi(k) sums behind every record (per ReLU warp, per feature)
+      const float4* zp = part4 + E4 + 2 * c_of[k];
+      for (int kk = 0; kk < nrec; ++kk) {
+        float4 w4[8][2];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+          w4[w][0] = __ldcg(zp + (size_t)record_of(kk) * REC4 + w * 32);
+          w4[w][1] = __ldcg(zp + (size_t)record_of(kk) * REC4 + w * 32 + 1);
+        }
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { add4(sum[k][0], w4[w][0]); add4(sum[k][1], w4[w][1]); }
+      }
+    }
+    const int j = j_of[k], c = c_of[k];
+    float4* dst = reinterpret_cast<float4*>(p.state) + (size_t)u * E4 + (size_t)j * (D / 4) + 2 * c;
+    dst[0] = sum[k][0];
+    dst[1] = sum[k][1];
+    const float x[8] = {sum[k][0].x, sum[k][0].y, sum[k][0].z, sum[k][0].w, sum[k][1].x, sum[k][1].y, sum[k][1].z, sum[k][1].w};
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
+      hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      lo[e] = pack_bf16x2(x[2 * e] - __bfloat162float(h0), x[2 * e + 1] - __bfloat162float(h1));
+    }
+    const int jrow = j < D ? j : C::ZROW;   // operand row: value feature, or the z row
+    const int i0 = c * 8;                   // first key feature of this chunk
+    const int off = (i0 >> 6) * C::SBOX_BYTES + jrow * kRowBytes + ((((i0 & 63) >> 3) ^ (jrow & 7)) << 4);
+    uint8_t* img = p.s_image + (size_t)u * C::S_BYTES;
+    *reinterpret_cast<uint4*>(img + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(img + 2 * C::SBOX_BYTES + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
+template <int D, bool ROPE>
+__device__ void reduce_image(const FusedParams& p) {
+  constexpr int TOTAL = (D + 1) * (D / 8);   // chunks of a unit
+  const Sched& s = p.sa;
+  const int me = (int)blockIdx.x;
+  if (me < s.P * s.U) {
+    const int u = me % s.U, c = me / s.U;
+    const int lo_i = c * TOTAL / s.P, hi_i = (c + 1) * TOTAL / s.P;
+    const int ncol = s.P < (s.tpu + s.Lc - 1) / s.Lc ? s.P : (s.tpu + s.Lc - 1) / s.Lc;
+    int r_lo = 0, ntrail = 0;
+    if (s.m > 0) {
+      const long long ttot = (long long)s.U * s.m;
+      r_lo = trailing_cta_of((long long)u * s.m, ttot, s.R);
+      ntrail = trailing_cta_of((long long)(u + 1) * s.m - 1, ttot, s.R) - r_lo + 1;
+    }
+    const int nrec = ncol + ntrail;
+    if (hi_i - lo_i <= (int)blockDim.x) {
+      reduce_image_chunks<D, ROPE, 1, ROPE ? 6 : 10>(p, u, lo_i + (int)threadIdx.x, hi_i, ncol, r_lo, nrec);
+    } else {
+      for (int first = lo_i + (int)threadIdx.x; first < hi_i; first += 2 * (int)blockDim.x)
+        reduce_image_chunks<D, ROPE, 2, ROPE ? 3 : 6>(p, u, first, hi_i, ncol, r_lo, nrec);
+    }
+  }
+  fence_proxy_async_all();   // the images are read through the async proxy (bulk copy) after the barrier
 }
 
 // ---------------------------------------------------------------- S operand of the apply pass
@@ -757,7 +877,10 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   // ==================================================================== reduce
   if (p.do_state) {
     grid_barrier(p.ctrl, abort_flag);
-    if (!*abort_flag) reduce_slice<D, ROPE>(p);
+    if (!*abort_flag) {
+      if (C::G == 1 && p.s_image) reduce_image<D, ROPE>(p);
+      else reduce_slice<D, ROPE>(p);
+    }
     if (p.do_apply) grid_barrier(p.ctrl, abort_flag);
   }
   if (C::G > 1 && wc.f1 > wc.f0) {
@@ -838,7 +961,17 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         if (seg > 0) ok = mbar_wait(seg_done, (seg - 1) & 1, abort_flag);
         if (!ok) break;
         const int u = t.unit();
-        build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, tr, R::RELU_THREADS + 128);
+        if (C::G == 1 && p.s_image) {
+          if (tr == 0) {   // the unit's operand image, made by the reduce: one bulk copy
+            fence_proxy_async_all();
+            mbar_arrive_expect_tx(s_ready, C::S_BYTES);
+            bulk_load(s_op, p.s_image + (size_t)u * C::S_BYTES, C::S_BYTES, s_ready);
+          } else {
+            mbar_arrive(s_ready);
+          }
+        } else {
+          build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, tr, R::RELU_THREADS + 128);
+        }
         if (ROPE) {
           const float4* zrow = reinterpret_cast<const float4*>(p.state + ((size_t)u * (D + 1) + D) * D);  // G = 1: unit = (b, h)
           const float4 a0 = __ldcg(zrow + 2 * lc), a1 = __ldcg(zrow + 2 * lc + 1);
@@ -848,8 +981,10 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
             zc[8] = b0.x; zc[9] = b0.y; zc[10] = b0.z; zc[11] = b0.w; zc[12] = b1.x; zc[13] = b1.y; zc[14] = b1.z; zc[15] = b1.w;
           }
         }
-        fence_proxy_async_smem();
-        mbar_arrive(s_ready);
+        if (!(C::G == 1 && p.s_image)) {
+          fence_proxy_async_smem();
+          mbar_arrive(s_ready);
+        }
         ++seg;
       }
       if (ROPE) {
@@ -902,8 +1037,10 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       if (t.seg_first()) {
         // this thread has seen the last accumulator of the previous segment complete: S may be rebuilt
         const int u = t.unit();
-        build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, R::RELU_THREADS + te, R::RELU_THREADS + 128);
-        fence_proxy_async_smem();
+        if (!(C::G == 1 && p.s_image)) {
+          build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, R::RELU_THREADS + te, R::RELU_THREADS + 128);
+          fence_proxy_async_smem();
+        }
         mbar_arrive(s_ready);
       }
       const uint32_t acc = it & 1;
@@ -1081,6 +1218,18 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   fp.ctrl = static_cast<WorkspaceCtrl*>(workspace);
   fp.rope = static_cast<const uint4*>(c.rope);
   fp.N = p.N;
+  fp.s_image = nullptr;
+  if (do_state && do_apply && C::G == 1 && fp.sa.P >= 1) {
+    // The operand images live at the end of the partials area, which is sized for kMaxCtas + U records while a
+    // launch writes at most P*U + R + U of them: used when they fit behind the records in use.
+    const size_t rec_bytes = ((size_t)p.state_elems() + (ROPE ? kZParts : 0)) * sizeof(float);
+    const size_t used = ((size_t)fp.sa.P * U + fp.sa.R + U) * rec_bytes;
+    const size_t total = umma_partial_bytes(p, ROPE), img = (size_t)U * C::S_BYTES;
+    if (total >= img + 1024) {
+      const size_t off = (total - img) & ~(size_t)1023;
+      if (off >= used) fp.s_image = reinterpret_cast<uint8_t*>(fp.partials) + off;
+    }
+  }
   int grid = 0;
   if (do_state) grid = fp.sa.grid;
   if (do_apply && fp.sc.grid > grid) grid = fp.sc.grid;
