@@ -230,3 +230,38 @@ def test_bounded_wait_reports_timeout_and_the_context_survives(la):
     la.load_library().linattn_workspace_init(ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
     assert la.workspace_status(ws) == 0
     assert torch.equal(la.linattn_state(k, v, workspace=ws), good)
+
+
+# Many units: how the persistent grid splits the work depends on the number of (batch, head) units U against
+# the 148 SMs.  U = 60: two column CTAs per unit plus trailing CTAs, operand images in use; U = 100: one column
+# CTA per unit plus trailing CTAs, images do not fit behind the records; U = 148: one CTA per unit, no trailing
+# CTAs; U = 200: more units than CTAs, every CTA walks over several units.
+@pytest.mark.parametrize("shape", [(3, 1500, 20, 112), (5, 700, 20, 112), (4, 600, 37, 112), (10, 400, 20, 112),
+                                   (3, 900, 18, 128)], ids=lambda s: "B%d_N%d_H%d_d%d" % s)
+def test_work_split_with_many_units(la, orc, shape):
+    import torch
+
+    B, N, H, d = shape
+    q, k, v = gen(B, N, H, d, 2300 + B * H, "bf16")
+    qd, kd, vd = to_dev(q), to_dev(k), to_dev(v)
+    ws = la.new_workspace(qd)
+    o = la.linattn_forward(qd, kd, vd, EPS, workspace=ws)
+    check("bf16", to_f64(o), orc.forward(q, k, v, EPS), f"forward {shape}")
+    assert torch.equal(o, la.linattn_forward(qd, kd, vd, EPS, workspace=ws))      # run-to-run determinism
+    # the fused launch and the two separate launches sum the same records in the same order
+    st = la.linattn_state(kd, vd, workspace=ws)
+    assert torch.equal(o, la.linattn_apply(qd, st, EPS))
+    # two cached steps over the halves: small integers make the cache exact, so both ways of reducing
+    # (on top of the old cache, with or without operand images) must give the oracle's bits
+    ki = synth.smallint((B, N, H, d), 2301, 2, 2)
+    vi = synth.smallint((B, N, H, d), 2301, 3, 2)
+    half = (N // 2 + 7) // 8 * 8
+    cache = la.BlockLinCache(B, H, d, torch.bfloat16, "cuda", max_T_b=half, eps=EPS)
+    outs = [cache.step(to_dev(np.ascontiguousarray(q[:, sl])), to_dev(np.ascontiguousarray(ki[:, sl])),
+                       to_dev(np.ascontiguousarray(vi[:, sl]))) for sl in (slice(0, half), slice(half, N))]
+    S, z = orc.state(ki, vi)
+    got = to_f64(cache.state)
+    assert np.array_equal(got[..., :d, :].swapaxes(-1, -2), S) and np.array_equal(got[..., d, :], z)
+    ref = orc.block_masked(q, ki, vi, EPS, half)
+    check("bf16", to_f64(torch.cat(outs, dim=1)), ref, f"two steps {shape}")
+    assert la.workspace_status(cache.workspace) == 0
