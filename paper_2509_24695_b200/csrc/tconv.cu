@@ -79,14 +79,14 @@ struct TconvParams {
   int D;
 };
 
-constexpr int kAhead = 3;   // frames in flight beyond the next one
-
-template <typename T>
-__global__ void __launch_bounds__(256, 3) tconv_kernel(const TconvParams p) {
+// kAhead: frames in flight beyond the next one.  Long clips run with 3 (79 registers, 3 blocks per SM); a block
+// step of up to three frames has all its frames in flight with 1 and fits 4 blocks per SM.
+template <typename T, int kAhead>
+__global__ void __launch_bounds__(256, kAhead > 1 ? 3 : 4) tconv_kernel(const TconvParams p) {
   using Pc = Piece<T>;
   using Raw = typename Pc::Raw;
   constexpr int PAIRS = Pc::PAIRS;
-  const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * (2 * PAIRS);   // element within a frame
+  const unsigned col = (blockIdx.x * blockDim.x + threadIdx.x) * (2 * PAIRS);   // element within a frame (< 2^31)
   if (col >= p.frame) return;
   const int b = blockIdx.y;
   const T* x = static_cast<const T*>(p.x) + b * p.sb + col;
@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(256, 3) tconv_kernel(const TconvParams p) {
   }
   T* y = static_cast<T*>(p.y) + b * p.sby + col;
 
-  const int c0 = (int)(col % p.D);
+  const int c0 = (int)(col % (unsigned)p.D);
   float2 w[3][PAIRS];
 #pragma unroll
   for (int tau = 0; tau < 3; ++tau)
@@ -151,6 +151,7 @@ int check(const tconv_desc* d, long long T, long long* frame, long long* sb, lon
   if (d->D % vec) return LINATTN_ERR_UNSUPPORTED;
   *esz = d->dtype == LINATTN_BF16 ? 2 : 4;
   *frame = (long long)d->HW * d->D;
+  if (*frame >= (1ll << 31)) return LINATTN_ERR_UNSUPPORTED;
   *sb = d->stride_b ? d->stride_b : T * *frame;
   *sby = d->stride_b_y ? d->stride_b_y : T * *frame;
   if (*sb % vec || *sby % vec) return LINATTN_ERR_BAD_ALIGNMENT;
@@ -185,8 +186,14 @@ int run(const tconv_desc* d, long long T, long long T_b, const void* x, const fl
   const int vec = d->dtype == LINATTN_BF16 ? 8 : 4;
   const long long cols = frame / vec;
   dim3 grid((unsigned)((cols + 255) / 256), (unsigned)d->B);
-  if (d->dtype == LINATTN_BF16) tconv_kernel<__nv_bfloat16><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
-  else tconv_kernel<float><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+  const bool few = T <= 3;
+  if (d->dtype == LINATTN_BF16) {
+    if (few) tconv_kernel<__nv_bfloat16, 1><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+    else tconv_kernel<__nv_bfloat16, 3><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+  } else {
+    if (few) tconv_kernel<float, 1><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+    else tconv_kernel<float, 3><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+  }
   count_launches(1);
   return cudaGetLastError() == cudaSuccess ? LINATTN_OK : LINATTN_ERR_CUDA;
 }
