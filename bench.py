@@ -481,6 +481,19 @@ def extras(torch, la, synth, dev, peak):
         res[w.name] = {"H": w.H, "d": w.d, "ms": ms, "tokens_heads_per_s": w.B * w.N * w.H / (ms * 1e-3),
                        "algorithmic_gbs": by / (ms * 1e-3) / 1e9, "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak,
                        "l2": "one input set of %.0f MB (> 126 MB L2)" % (by / 1e6)}
+        if w.d == 112:
+            # the same layer with head-major memory ([B,H,N,d] behind the same [B,N,H,d] view): a head's rows are
+            # then contiguous instead of 224 bytes out of every 4480
+            hm = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+            qh, kh, vh = hm(q), hm(k), hm(v)
+            oh = hm(o)
+            wsh = la.new_workspace(qh)
+            for _ in range(3):
+                la.linattn_forward(qh, kh, vh, w.eps, out=oh, workspace=wsh)
+            ms = time_loop(torch, lambda i: la.linattn_forward(qh, kh, vh, w.eps, out=oh, workspace=wsh), n) / n
+            res[w.name + "_head_major"] = {"H": w.H, "d": w.d, "ms": ms, "layout": "[B,H,N,d] memory (strides in the descriptor)",
+                                           "algorithmic_gbs": by / (ms * 1e-3) / 1e9, "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak}
+            del qh, kh, vh, oh, wsh
         del q, k, v, o, ws
     # Eq. 2 with its rotary factors on the 480p layer (3D table over the 21 x 30 x 52 latent grid)
     w = synth.P480
