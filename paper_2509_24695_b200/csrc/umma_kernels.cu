@@ -236,21 +236,22 @@ __device__ __forceinline__ void relu_pass(uint8_t* box0, uint8_t* box1, int t) {
 
 // Rotary variant: a 16-byte chunk holds four feature pairs; `tab` holds their (cos, sin) as fp16 pairs.
 // (a, b) -> (a c - b s, a s + b c), rounded to bf16.
-__device__ __forceinline__ void unpack_relu8(const uint4& x, float (&f)[8]) {
-  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+// The ReLU role of the rotary variant is bound by instruction issue, so the clamp is done on the packed bf16
+// pairs and the sums, the rotation and the denominators use the packed f32x2 instructions.
+__device__ __forceinline__ void unpack_relu8(const uint4& x, float2 (&f)[4]) {
+  const uint32_t w[4] = {relu_bf16x2(x.x), relu_bf16x2(x.y), relu_bf16x2(x.z), relu_bf16x2(x.w)};
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    f[2 * e] = fmaxf(__uint_as_float(w[e] << 16), 0.f);
-    f[2 * e + 1] = fmaxf(__uint_as_float(w[e] & 0xFFFF0000u), 0.f);
-  }
+  for (int e = 0; e < 4; ++e) f[e] = make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xFFFF0000u));
 }
-__device__ __forceinline__ uint4 rotate_pack8(const float (&f)[8], const uint4& tab) {
+__device__ __forceinline__ uint4 rotate_pack8(const float2 (&f)[4], const uint4& tab) {
   const uint32_t t[4] = {tab.x, tab.y, tab.z, tab.w};
   uint32_t o[4];
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
     const float2 cs = __half22float2(*reinterpret_cast<const __half2*>(&t[e]));
-    o[e] = pack_bf16x2(f[2 * e] * cs.x - f[2 * e + 1] * cs.y, f[2 * e] * cs.y + f[2 * e + 1] * cs.x);
+    // (a, b) -> (a c - b s, b c + a s) = (-b, a) * (s, s) + (a, b) * (c, c)
+    const float2 r = fma2(make_float2(-f[e].y, f[e].x), make_float2(cs.y, cs.y), mul2(f[e], make_float2(cs.x, cs.x)));
+    o[e] = pack_bf16x2(r.x, r.y);
   }
   return make_uint4(o[0], o[1], o[2], o[3]);
 }
@@ -726,9 +727,9 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     // rotary variant: this thread's 16-byte column holds logical chunk lc of every row it touches
     const int row0 = tr >> 3, pc = tr & 7, lc = pc ^ (row0 & 7);
     const bool box1_live = 64 + lc * 8 < C::FEAT;
-    float zacc[16];  // sums of the plain phi(k) over the segment: features 8*lc.. of box 0, 64 + 8*lc.. of box 1
+    float2 zacc[8];  // sums of the plain phi(k) over the segment: features 8*lc.. of box 0, 64 + 8*lc.. of box 1
 #pragma unroll
-    for (int e = 0; e < 16; ++e) zacc[e] = 0.f;
+    for (int e = 0; e < 8; ++e) zacc[e] = make_float2(0.f, 0.f);
     // The rotations of a row do not depend on K: they are fetched one stage ahead, each register reloaded
     // for the next stage right after its use, so that their latency is off the stage's critical path.
     uint4 tab0[kTileState / 32], tab1[kTileState / 32];
@@ -757,17 +758,17 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         uint8_t* p0 = st + C::KOFF + row0 * kRowBytes + pc * 16;
 #pragma unroll
         for (int i = 0; i < kTileState / 32; ++i) {
-          float f[8];
+          float2 f[4];
           uint4* c0 = reinterpret_cast<uint4*>(p0 + i * 32 * kRowBytes);
           unpack_relu8(*c0, f);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) zacc[e] += f[e];
+          for (int e = 0; e < 4; ++e) zacc[e] = add2(zacc[e], f[e]);
           *c0 = rotate_pack8(f, tab0[i]);
           if (box1_live) {
             uint4* c1 = reinterpret_cast<uint4*>(p0 + kBox + i * 32 * kRowBytes);
             unpack_relu8(*c1, f);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) zacc[8 + e] += f[e];
+            for (int e = 0; e < 4; ++e) zacc[4 + e] = add2(zacc[4 + e], f[e]);
             *c1 = rotate_pack8(f, tab1[i]);
           }
           if (!tn.done()) fetch_rot(tn.tile(), i);
@@ -785,7 +786,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
           for (int rr = 0; rr < 4; ++rr) {
             const int src = (rr << 3) | (lc ^ ((4 * (w & 1) + rr) & 7));
 #pragma unroll
-            for (int e = 0; e < 16; ++e) tot[e] += __shfl_sync(0xffffffffu, zacc[e], src);
+            for (int e = 0; e < 16; ++e) tot[e] += __shfl_sync(0xffffffffu, (e & 1) ? zacc[e >> 1].y : zacc[e >> 1].x, src);
           }
           if (r == 0) {
             float* zp = p.partials + (size_t)t.record() * (C::G * (D + 1) * D + kZParts) + C::G * (D + 1) * D + w * 128;
@@ -797,7 +798,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
             }
           }
 #pragma unroll
-          for (int e = 0; e < 16; ++e) zacc[e] = 0.f;
+          for (int e = 0; e < 8; ++e) zacc[e] = make_float2(0.f, 0.f);
         }
         continue;
       }
@@ -934,9 +935,9 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     // rotary variant: this thread's 16-byte column holds logical chunk lc of every row it touches
     const int row0 = tr >> 3, pc = tr & 7, lc = pc ^ (row0 & 7);
     const bool box1_live = 64 + lc * 8 < C::FEAT;
-    float zc[16];  // the segment's z at this thread's features (8*lc.. of box 0, 64 + 8*lc.. of box 1)
+    float2 zc[8];  // the segment's z at this thread's features (8*lc.. of box 0, 64 + 8*lc.. of box 1)
 #pragma unroll
-    for (int e = 0; e < 16; ++e) zc[e] = 0.f;
+    for (int e = 0; e < 8; ++e) zc[e] = make_float2(0.f, 0.f);
     // rotations one tile ahead, as in the state pass
     uint4 tab0[kTileApply / 32], tab1[kTileApply / 32];
     auto fetch_rot = [&](int tile, int i) {
@@ -975,10 +976,10 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         if (ROPE) {
           const float4* zrow = reinterpret_cast<const float4*>(p.state + ((size_t)u * (D + 1) + D) * D);  // G = 1: unit = (b, h)
           const float4 a0 = __ldcg(zrow + 2 * lc), a1 = __ldcg(zrow + 2 * lc + 1);
-          zc[0] = a0.x; zc[1] = a0.y; zc[2] = a0.z; zc[3] = a0.w; zc[4] = a1.x; zc[5] = a1.y; zc[6] = a1.z; zc[7] = a1.w;
+          zc[0] = make_float2(a0.x, a0.y); zc[1] = make_float2(a0.z, a0.w); zc[2] = make_float2(a1.x, a1.y); zc[3] = make_float2(a1.z, a1.w);
           if (box1_live) {
             const float4 b0 = __ldcg(zrow + 16 + 2 * lc), b1 = __ldcg(zrow + 16 + 2 * lc + 1);
-            zc[8] = b0.x; zc[9] = b0.y; zc[10] = b0.z; zc[11] = b0.w; zc[12] = b1.x; zc[13] = b1.y; zc[14] = b1.z; zc[15] = b1.w;
+            zc[4] = make_float2(b0.x, b0.y); zc[5] = make_float2(b0.z, b0.w); zc[6] = make_float2(b1.x, b1.y); zc[7] = make_float2(b1.z, b1.w);
           }
         }
         if (!(C::G == 1 && p.s_image)) {
@@ -997,20 +998,21 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         uint8_t* p0 = sl + row0 * kRowBytes + pc * 16;
 #pragma unroll
         for (int i = 0; i < kTileApply / 32; ++i) {
-          float f[8];
+          float2 f[4];
           uint4* c0 = reinterpret_cast<uint4*>(p0 + i * 32 * kRowBytes);
           unpack_relu8(*c0, f);
-          float den = 0.f;
+          float2 den2 = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) den = fmaf(f[e], zc[e], den);
+          for (int e = 0; e < 4; ++e) den2 = fma2(f[e], zc[e], den2);
           *c0 = rotate_pack8(f, tab0[i]);
           uint4* c1 = reinterpret_cast<uint4*>(p0 + HALF + i * 32 * kRowBytes);
           if (box1_live) {
             unpack_relu8(*c1, f);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) den = fmaf(f[e], zc[8 + e], den);
+            for (int e = 0; e < 4; ++e) den2 = fma2(f[e], zc[4 + e], den2);
             *c1 = rotate_pack8(f, tab1[i]);
           }
+          float den = den2.x + den2.y;
           if (!tn.done()) fetch_rot(tn.tile(), i);  // this row's rotations for the next tile
           den += __shfl_xor_sync(0xffffffffu, den, 1);
           den += __shfl_xor_sync(0xffffffffu, den, 2);
