@@ -365,16 +365,24 @@ __device__ __forceinline__ void reduce_elements(const FusedParams& p, int first,
     const int idx = first + k * (int)blockDim.x;
     if (ROPE && zpart[k]) {
       // rotary variant: z comes from the plain phi(k) sums that the ReLU warps of every segment left
-      // behind the record (per warp, per feature); records in their fixed order, warps 0..7 within each
+      // behind the record (per warp, per feature): per warp slot the records in their fixed order, then the
+      // eight slots as a balanced tree (the association reduce_image's shuffles give)
       const int e = idx % E4;
       const float4* zp = reinterpret_cast<const float4*>(p.partials) + E4 + (e - D * D / 4);
-      for (int kk = 0; kk < nrec[k]; ++kk) {
-        float4 w4[8];
+      // (one slot after the other: this form only runs when the operand images are not in use, and the
+      // rotary kernel has no registers to spare)
+      float4 acc[8];
 #pragma unroll
-        for (int w = 0; w < 8; ++w) w4[w] = __ldcg(zp + (size_t)record_of(k, kk) * REC4 + w * 32);
-#pragma unroll
-        for (int w = 0; w < 8; ++w) add4(sum[k], w4[w]);
+      for (int w = 0; w < 8; ++w) {
+        acc[w] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+        for (int kk = 0; kk < nrec[k]; ++kk) add4(acc[w], __ldcg(zp + (size_t)record_of(k, kk) * REC4 + w * 32));
       }
+#pragma unroll
+      for (int st = 1; st < 8; st *= 2)
+#pragma unroll
+        for (int w = 0; w < 8; w += 2 * st) add4(acc[w], acc[w + st]);
+      add4(sum[k], acc[0]);
     }
     state4[idx] = sum[k];
   }
@@ -429,7 +437,7 @@ __device__ __forceinline__ void reduce_image_chunks(const FusedParams& p, int u,
     if (!live[k]) continue;
     j_of[k] = idx / CPR;
     c_of[k] = idx - j_of[k] * CPR;
-    zrow[k] = ROPE && j_of[k] == D;
+    zrow[k] = false;   // (rotary variant: the z row is not among the chunks, see reduce_image_zrow)
     const size_t e4 = (size_t)u * E4 + (size_t)j_of[k] * (D / 4) + 2 * c_of[k];
     if (p.accumulate) {
       sum[k][0] = __ldcg(reinterpret_cast<const float4*>(p.state_base) + e4);
@@ -457,20 +465,6 @@ __device__ __forceinline__ void reduce_image_chunks(const FusedParams& p, int u,
 #pragma unroll
   for (int k = 0; k < NE; ++k) {
     if (!live[k]) continue;
-    if (ROPE && zrow[k]) {
-      // rotary variant: z from the plain phi(k) sums behind every record (per ReLU warp, per feature)
-      const float4* zp = part4 + E4 + 2 * c_of[k];
-      for (int kk = 0; kk < nrec; ++kk) {
-        float4 w4[8][2];
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {
-          w4[w][0] = __ldcg(zp + (size_t)record_of(kk) * REC4 + w * 32);
-          w4[w][1] = __ldcg(zp + (size_t)record_of(kk) * REC4 + w * 32 + 1);
-        }
-#pragma unroll
-        for (int w = 0; w < 8; ++w) { add4(sum[k][0], w4[w][0]); add4(sum[k][1], w4[w][1]); }
-      }
-    }
     const int j = j_of[k], c = c_of[k];
     float4* dst = reinterpret_cast<float4*>(p.state) + (size_t)u * E4 + (size_t)j * (D / 4) + 2 * c;
     dst[0] = sum[k][0];
@@ -492,9 +486,65 @@ __device__ __forceinline__ void reduce_image_chunks(const FusedParams& p, int u,
   }
 }
 
+// Rotary variant: z of unit u from the plain phi(k) sums that the ReLU warps of every segment left behind the
+// record, [8 warp slots][128 features].  Thread (float4 hc of z, slot w) adds its slot over the records in their
+// fixed order (all loads in flight together), shuffles add the eight slots as a balanced tree, lane w = 0 adds
+// the old z when accumulating; two neighbouring float4 make the 32-byte chunk of the operand image.
+template <int D>
+__device__ __forceinline__ void reduce_image_zrow(const FusedParams& p, int u, int ncol, int r_lo, int nrec) {
+  using C = Cfg<D>;
+  constexpr int E4 = (D + 1) * D / 4, REC4 = E4 + kZParts / 4, Z4 = D / 4, NR = 6;
+  static_assert((8 * Z4) % 32 == 0 && Z4 % 2 == 0, "whole warps take part in the shuffles");
+  const int t = (int)threadIdx.x;
+  if (t >= 8 * Z4) return;
+  const int hc = t >> 3, w = t & 7;
+  const Sched& s = p.sa;
+  auto record_of = [&](int kk) { return kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u; };
+  const float4* zp = reinterpret_cast<const float4*>(p.partials) + E4 + w * 32 + hc;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int k0 = 0; k0 < nrec; k0 += NR) {
+    float4 v[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r)
+      if (k0 + r < nrec) v[r] = __ldcg(zp + (size_t)record_of(k0 + r) * REC4);
+#pragma unroll
+    for (int r = 0; r < NR; ++r)
+      if (k0 + r < nrec) add4(acc, v[r]);
+  }
+#pragma unroll
+  for (int st = 1; st < 8; st *= 2) {
+    float4 o;
+    o.x = __shfl_xor_sync(0xffffffffu, acc.x, st); o.y = __shfl_xor_sync(0xffffffffu, acc.y, st);
+    o.z = __shfl_xor_sync(0xffffffffu, acc.z, st); o.w = __shfl_xor_sync(0xffffffffu, acc.w, st);
+    add4(acc, o);
+  }
+  const size_t e4 = (size_t)u * E4 + (size_t)D * (D / 4) + hc;
+  float4 sum = p.accumulate ? __ldcg(reinterpret_cast<const float4*>(p.state_base) + e4) : make_float4(0.f, 0.f, 0.f, 0.f);
+  add4(sum, acc);
+  float4 up;   // the upper half of this chunk, from the lane that holds float4 hc + 1
+  up.x = __shfl_xor_sync(0xffffffffu, sum.x, 8); up.y = __shfl_xor_sync(0xffffffffu, sum.y, 8);
+  up.z = __shfl_xor_sync(0xffffffffu, sum.z, 8); up.w = __shfl_xor_sync(0xffffffffu, sum.w, 8);
+  if (w != 0) return;
+  reinterpret_cast<float4*>(p.state)[e4] = sum;
+  if (hc & 1) return;
+  const float x[8] = {sum.x, sum.y, sum.z, sum.w, up.x, up.y, up.z, up.w};
+  uint32_t hi[4], lo[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
+    hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+    lo[e] = pack_bf16x2(x[2 * e] - __bfloat162float(h0), x[2 * e + 1] - __bfloat162float(h1));
+  }
+  const int jrow = C::ZROW, i0 = (hc >> 1) * 8;
+  const int off = (i0 >> 6) * C::SBOX_BYTES + jrow * kRowBytes + ((((i0 & 63) >> 3) ^ (jrow & 7)) << 4);
+  uint8_t* img = p.s_image + (size_t)u * C::S_BYTES;
+  *reinterpret_cast<uint4*>(img + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+  *reinterpret_cast<uint4*>(img + 2 * C::SBOX_BYTES + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+}
+
 template <int D, bool ROPE>
 __device__ void reduce_image(const FusedParams& p) {
-  constexpr int TOTAL = (D + 1) * (D / 8);   // chunks of a unit
+  constexpr int TOTAL = (D + (ROPE ? 0 : 1)) * (D / 8);   // chunks of a unit (rotary: the z row goes separately)
   const Sched& s = p.sa;
   const int me = (int)blockIdx.x;
   if (me < s.P * s.U) {
@@ -514,6 +564,7 @@ __device__ void reduce_image(const FusedParams& p) {
       for (int first = lo_i + (int)threadIdx.x; first < hi_i; first += 2 * (int)blockDim.x)
         reduce_image_chunks<D, ROPE, 2, ROPE ? 3 : 6>(p, u, first, hi_i, ncol, r_lo, nrec);
     }
+    if (ROPE && D % 8 == 0 && c == 0) reduce_image_zrow<D>(p, u, ncol, r_lo, nrec);
   }
   fence_proxy_async_all();   // the images are read through the async proxy (bulk copy) after the barrier
 }
