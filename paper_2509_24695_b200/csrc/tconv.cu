@@ -142,6 +142,126 @@ __global__ void __launch_bounds__(256, kAhead > 1 ? 3 : 4) tconv_kernel(const Tc
   if (cache_out) *cache_out = Pc::pack(fp);   // fp is now the last frame; packing widened elements is exact
 }
 
+// Block steps of up to three frames (the paper's blocks are three latent frames).  Here a thread's share is only
+// four 16-byte loads (the cached frame and the block's frames), so what bounds the kernel is how many bytes an
+// SM keeps in flight, and registers are the wrong place to hold them: each thread streams its pieces into a
+// private ring in shared memory with cp.async (no registers held, nothing to poll: cp.async.wait_group is a
+// hardware wait), three tiles deep, and a persistent grid of four CTAs per SM walks the tiles (measured: threads
+// matter more than depth; 3 x 4 beat 6 x 2 by 12 % and 12 x 1 by 35 %; five CTAs per SM spill).  A tile is 256
+// consecutive 16-byte pieces of one batch entry's frame; no data is shared between threads, so no CTA-wide
+// synchronisation is needed.  Same arithmetic, in the same order, as tconv_kernel: the results are the same bits.
+constexpr int kStepStages = 3;
+constexpr int kStepSegs = 4;   // cached frame + up to three frames
+constexpr int kStepCtasPerSm = 4;
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <typename T>
+__global__ void __launch_bounds__(256, kStepCtasPerSm) tconv_step_kernel(const TconvParams p, int tiles_per_batch, int total_tiles) {
+  using Pc = Piece<T>;
+  using Raw = typename Pc::Raw;
+  constexpr int PAIRS = Pc::PAIRS;
+  extern __shared__ uint4 ring_raw[];
+  Raw* ring = reinterpret_cast<Raw*>(ring_raw);   // [stage][segment][thread]
+  const int tid = (int)threadIdx.x;
+  const int nf = (int)p.T;                        // 1..3 frames
+  auto locate = [&](int tile, int& b, unsigned& col) {
+    b = tile / tiles_per_batch;
+    col = (unsigned)((tile - b * tiles_per_batch) * 256 + tid) * (2 * PAIRS);
+  };
+  auto issue = [&](int tile, int stage) {
+    if (tile < total_tiles) {
+      int b;
+      unsigned col;
+      locate(tile, b, col);
+      if (col < p.frame) {
+        Raw* dst = ring + (stage * kStepSegs) * 256 + tid;
+        cp_async16(dst, static_cast<const T*>(p.cache_in) + (long long)b * p.frame + col);
+        const T* x = static_cast<const T*>(p.x) + b * p.sb + col;
+        for (int t = 0; t < nf; ++t) cp_async16(dst + (1 + t) * 256, x + t * p.frame);
+      }
+    }
+    cp_async_commit();   // one group per tile, empty or not, so that the count below stays uniform
+  };
+  const int first = (int)blockIdx.x, step = (int)gridDim.x;
+#pragma unroll
+  for (int s = 0; s < kStepStages - 1; ++s) issue(first + s * step, s);
+  int k = 0;
+  for (int tile = first; tile < total_tiles; tile += step, ++k) {
+    issue(tile + (kStepStages - 1) * step, (k + kStepStages - 1) % kStepStages);
+    cp_async_wait<kStepStages - 1>();   // this thread's copies of `tile` have landed
+    int b;
+    unsigned col;
+    locate(tile, b, col);
+    if (col >= p.frame) continue;
+    const int c0 = (int)(col % (unsigned)p.D);
+    float2 w[3][PAIRS];
+#pragma unroll
+    for (int tau = 0; tau < 3; ++tau)
+#pragma unroll
+      for (int i = 0; i < PAIRS; i += 2) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(p.w + tau * p.D + c0 + 2 * i));
+        w[tau][i] = make_float2(a.x, a.y);
+        w[tau][i + 1] = make_float2(a.z, a.w);
+      }
+    const Raw* src = ring + ((k % kStepStages) * kStepSegs) * 256 + tid;
+    float2 fp[PAIRS], fc[PAIRS], fn[PAIRS];
+    Pc::unpack(src[0], fp);
+    Pc::unpack(src[256], fc);
+    T* y = static_cast<T*>(p.y) + b * p.sby + col;
+    for (int t = 0; t < nf; ++t) {
+      const bool last = t + 1 == nf;
+      if (!last) Pc::unpack(src[(2 + t) * 256], fn);
+      float2 fo[PAIRS];
+#pragma unroll
+      for (int i = 0; i < PAIRS; ++i) fo[i] = fma2(w[1][i], fc[i], fma2(w[0][i], fp[i], fc[i]));
+      if (!last) {
+#pragma unroll
+        for (int i = 0; i < PAIRS; ++i) fo[i] = fma2(w[2][i], fn[i], fo[i]);
+      }
+      __stcs(reinterpret_cast<Raw*>(y + t * p.frame), Pc::pack(fo));
+#pragma unroll
+      for (int i = 0; i < PAIRS; ++i) { fp[i] = fc[i]; fc[i] = fn[i]; }
+    }
+    if (p.cache_out)   // fp is now the block's last frame
+      *reinterpret_cast<Raw*>(static_cast<T*>(p.cache_out) + (long long)b * p.frame + col) = Pc::pack(fp);
+  }
+  cp_async_wait<0>();
+}
+
+int sm_count_of_device() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return 0;
+  return n;
+}
+
+template <typename T>
+cudaError_t launch_step(const TconvParams& p, int B, cudaStream_t stream) {
+  constexpr int vec = 2 * Piece<T>::PAIRS;
+  const long long cols = p.frame / vec;
+  const long long tpb = (cols + 255) / 256, total = tpb * B;
+  if (total >= (1ll << 31)) return cudaErrorInvalidValue;
+  constexpr size_t smem = (size_t)kStepStages * kStepSegs * 256 * 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    const cudaError_t e = cudaFuncSetAttribute(tconv_step_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int sms = sm_count_of_device();
+  if (!sms) return cudaErrorUnknown;
+  const int grid = (int)(total < kStepCtasPerSm * sms ? total : kStepCtasPerSm * sms);
+  tconv_step_kernel<T><<<grid, 256, smem, stream>>>(p, (int)tpb, (int)total);
+  return cudaGetLastError();
+}
+
 int check(const tconv_desc* d, long long T, long long* frame, long long* sb, long long* sby, size_t* esz) {
   if (!d || T < 0) return LINATTN_ERR_INVALID_ARG;
   if (d->B < 1 || d->HW < 1 || d->D < 1 || d->stride_b < 0 || d->stride_b_y < 0) return LINATTN_ERR_INVALID_ARG;
@@ -187,15 +307,22 @@ int run(const tconv_desc* d, long long T, long long T_b, const void* x, const fl
   const long long cols = frame / vec;
   dim3 grid((unsigned)((cols + 255) / 256), (unsigned)d->B);
   const bool few = T <= 3;
-  if (d->dtype == LINATTN_BF16) {
-    if (few) tconv_kernel<__nv_bfloat16, 1><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
-    else tconv_kernel<__nv_bfloat16, 3><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+  cudaError_t e;
+  if (few && cache_in && y) {   // a block step of the paper's size: the staged kernel
+    e = d->dtype == LINATTN_BF16 ? launch_step<__nv_bfloat16>(p, d->B, (cudaStream_t)stream)
+                                 : launch_step<float>(p, d->B, (cudaStream_t)stream);
   } else {
-    if (few) tconv_kernel<float, 1><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
-    else tconv_kernel<float, 3><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+    if (d->dtype == LINATTN_BF16) {
+      if (few) tconv_kernel<__nv_bfloat16, 1><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+      else tconv_kernel<__nv_bfloat16, 3><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+    } else {
+      if (few) tconv_kernel<float, 1><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+      else tconv_kernel<float, 3><<<grid, 256, 0, (cudaStream_t)stream>>>(p);
+    }
+    e = cudaGetLastError();
   }
   count_launches(1);
-  return cudaGetLastError() == cudaSuccess ? LINATTN_OK : LINATTN_ERR_CUDA;
+  return e == cudaSuccess ? LINATTN_OK : LINATTN_ERR_CUDA;
 }
 
 }  // namespace
