@@ -924,6 +924,19 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       mbar_arrive(a_tempty);
       ++seg;
     }
+  } else if (C::G == 1 && p.s_image && p.accumulate && p.do_state && (int)blockIdx.x < p.sa.P * p.sa.U) {
+    // ------------------------------------------------------------ store warp (idle in this pass)
+    // A cached step adds to the old state, which the K, V stream has pushed out of L2 since the last step:
+    // once this CTA's loads are all issued, ask for its share of it (reduce_image's split), so that the
+    // reduce finds it in L2 instead of waiting for DRAM between the two grid barriers.
+    if (__all_sync(0xffffffffu, mbar_wait(a_done, 0, abort_flag))) {
+      constexpr int TOTAL = (D + (ROPE ? 0 : 1)) * (D / 8);
+      const int u = (int)blockIdx.x % p.sa.U, c = (int)blockIdx.x / p.sa.U;
+      const int lo_i = c * TOTAL / p.sa.P, hi_i = (c + 1) * TOTAL / p.sa.P;
+      const char* base = reinterpret_cast<const char*>(p.state_base + (size_t)u * ((D + 1) * D)) + (size_t)lo_i * 32;
+      for (int off = lane * 128; off < (hi_i - lo_i) * 32; off += 32 * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off) : "memory");
+    }
   }
 
   // ==================================================================== reduce
@@ -1262,7 +1275,7 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   fp.B = p.B; fp.H = p.H; fp.HG = (p.H + C::G - 1) / C::G;
   const int U = p.B * fp.HG;
   fp.sa = make_sched(U, (p.N + kTileState - 1) / kTileState, sms, 2);
-  fp.sc = make_sched(U, (p.N + kTileApply - 1) / kTileApply, sms, 2);
+  fp.sc = make_sched(U, (p.N + kTileApply - 1) / kTileApply, sms, 1);  // a unit switch costs the apply pass about one tile
   fp.do_state = do_state; fp.do_apply = do_apply; fp.accumulate = c.accumulate ? 1 : 0;
   fp.state = c.state;
   fp.state_base = c.state_base ? c.state_base : c.state;
