@@ -32,7 +32,7 @@
  *   functions oracle_rope_*).  The paper fixes neither how features are paired
  *   nor the angles: pairs are adjacent features and the rotations are inputs.
  *
- * Readings taken where the paper is silent (each is listed in the design doc):
+ * Readings taken where the paper is silent:
  *   - eps is added once to the denominator after the dot product;
  *   - a query whose phi(q).z is zero yields 0/(0+eps) = 0, never NaN;
  *   - "D" in the O(D^2) cache size is the per-head dimension d;
