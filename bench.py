@@ -276,7 +276,7 @@ def main():
     # alone (same kernel, one pass switched off), for reference.
     state_buf = la.linattn_state(sets[0][1], sets[0][2], workspace=ws)
     ms_state = time_loop(torch, lambda i: la.linattn_state(sets[i & 1][1], sets[i & 1][2], out=state_buf, workspace=ws), K) / K
-    ms_apply = time_loop(torch, lambda i: la.linattn_apply(sets[i & 1][0], state_buf, w.eps, out=sets[i & 1][3]), K) / K
+    ms_apply = time_loop(torch, lambda i: la.linattn_apply(sets[i & 1][0], state_buf, w.eps, out=sets[i & 1][3], workspace=ws), K) / K
     peak, peak_kind = peaks()
     bytes_tok_head = 2 * w.d  # one bf16 row of d features
     state_bytes = la.state_bytes(w.B, w.H, w.d)

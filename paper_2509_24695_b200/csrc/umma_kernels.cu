@@ -1275,7 +1275,6 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   fp.B = p.B; fp.H = p.H; fp.HG = (p.H + C::G - 1) / C::G;
   const int U = p.B * fp.HG;
   fp.sa = make_sched(U, (p.N + kTileState - 1) / kTileState, sms, 2);
-  fp.sc = make_sched(U, (p.N + kTileApply - 1) / kTileApply, sms, 1);  // a unit switch costs the apply pass about one tile
   fp.do_state = do_state; fp.do_apply = do_apply; fp.accumulate = c.accumulate ? 1 : 0;
   fp.state = c.state;
   fp.state_base = c.state_base ? c.state_base : c.state;
@@ -1296,6 +1295,9 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
       if (off >= used) fp.s_image = reinterpret_cast<uint8_t*>(fp.partials) + off;
     }
   }
+  // a unit switch costs the apply pass about one tile when the S operand comes as an image, two when the CTA
+  // builds it from the fp32 state
+  fp.sc = make_sched(U, (p.N + kTileApply - 1) / kTileApply, sms, fp.s_image ? 1 : 2);
   int grid = 0;
   if (do_state) grid = fp.sa.grid;
   if (do_apply && fp.sc.grid > grid) grid = fp.sc.grid;
