@@ -102,3 +102,20 @@ def test_tconv_sizes_and_validation_without_gpu(lib):
     assert lib.tconv_forward(ctypes.byref(d), -1, None, None, None, None) == -1
     assert lib.tconv_block_step(ctypes.byref(d), 3, None, None, None, None, 1, None) == -1
     assert lib.tconv_prefill(ctypes.byref(d), -1, 3, None, None, None, None, None) == -1
+
+
+def test_prefill_workspace_size_without_gpu(lib):
+    """Room for taking all blocks of a prefill together: never less than what single steps need, grows with the
+    number of blocks (one more set of per-block states and records each), refuses what the grid cannot index."""
+    import paper_2509_24695_b200 as la
+
+    d = la._Desc(1, 20, 112, 0, 0, 0, 0)
+    step_state, step_ws, pre = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()
+    assert lib.blocklin_cache_bytes(ctypes.byref(d), 4680, ctypes.byref(step_state), ctypes.byref(step_ws)) == 0
+    assert lib.blocklin_prefill_workspace_bytes(ctypes.byref(d), 1, 4680, ctypes.byref(pre)) == 0
+    one = pre.value
+    assert lib.blocklin_prefill_workspace_bytes(ctypes.byref(d), 7, 4680, ctypes.byref(pre)) == 0
+    assert pre.value > one and pre.value >= 7 * step_state.value and pre.value % 256 == 0
+    assert lib.blocklin_prefill_workspace_bytes(ctypes.byref(d), 4000, 4680, ctypes.byref(pre)) == -2   # 80 000 units
+    assert lib.blocklin_prefill_workspace_bytes(ctypes.byref(d), 0, 4680, ctypes.byref(pre)) == -1
+    assert lib.blocklin_prefill_workspace_bytes(ctypes.byref(d), 7, 4680, None) == -1
