@@ -264,26 +264,32 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
   return v;
 }
 
-// All CTAs of the (cooperatively launched, hence co-resident) grid meet here.  One word holds the
-// arrival count (low 16 bits) and a generation (high 16 bits): the last CTA to arrive clears the count
-// and bumps the generation with one more atomic, the others poll the word until the generation
-// moves.  The poll is bounded (about a second); on expiry the CTA raises its abort flag and goes on to
-// the teardown.
-__device__ __forceinline__ void grid_barrier(WorkspaceCtrl* ctrl, volatile int* abort_flag) {
+// All CTAs of the (cooperatively launched, hence co-resident) grid meet here.  One word holds an arrival count
+// (low 16 bits) and a generation (high 16 bits).  Before a barrier the count is pre-set to 2^16 - grid (CTA 0 adds
+// that: at kernel start for the first barrier, on leaving a barrier for the next one), so the last arrival's own
+// atomic add carries into the generation: the CTAs polling the word see the barrier open one L2 round trip after
+// the last arrival, with no second, dependent atomic in between (that cost 0.6 us per barrier).  All updates are
+// atomic adds, which commute, so the carry happens at the (grid + 1)-th add whatever their order, and the count is
+// back at zero after the launch's last barrier.  The poll is bounded (about a second); on expiry the CTA raises
+// its abort flag and goes on to the teardown.
+__device__ __forceinline__ void grid_barrier_preset(WorkspaceCtrl* ctrl) {
+  atomicAdd(&ctrl->barrier[0], 0x10000u - gridDim.x);
+}
+
+__device__ __forceinline__ void grid_barrier(WorkspaceCtrl* ctrl, volatile int* abort_flag, bool another_follows) {
   tcgen05_fence_before();
   __syncthreads();
   if (threadIdx.x == 0) {
     unsigned* word = &ctrl->barrier[0];
     __threadfence();
     const unsigned old = atomicAdd(word, 1u);
-    if ((old & 0xFFFFu) == gridDim.x - 1) {
-      atomicAdd(word, 0x10000u - gridDim.x);
-    } else {
+    if ((old & 0xFFFFu) != 0xFFFFu) {   // not the arrival that opened it
       const unsigned long long t0 = global_timer_ns();
       while ((ld_acquire_gpu(word) >> 16) == (old >> 16)) {
         if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
       }
     }
+    if (another_follows && blockIdx.x == 0 && !*abort_flag) grid_barrier_preset(ctrl);
     __threadfence();
   }
   __syncthreads();
@@ -666,6 +672,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   const Work wc = p.do_apply ? work_of(p.sc, blockIdx.x) : work_of(p.sc, 0x7fffffff);
 
   if (threadIdx.x == 0) {
+    if (blockIdx.x == 0 && p.do_state) grid_barrier_preset(p.ctrl);   // for the first grid barrier
     for (int s = 0; s < NSA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_ready[s], R::RELU_THREADS); mbar_init(&a_empty[s], 1); }
     mbar_init(a_tfull, 1);
     mbar_init(a_tempty, 128);
@@ -941,12 +948,12 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 
   // ==================================================================== reduce
   if (p.do_state) {
-    grid_barrier(p.ctrl, abort_flag);
+    grid_barrier(p.ctrl, abort_flag, p.do_apply != 0);
     if (!*abort_flag) {
       if (C::G == 1 && p.s_image) reduce_image<D, ROPE>(p);
       else reduce_slice<D, ROPE>(p);
     }
-    if (p.do_apply) grid_barrier(p.ctrl, abort_flag);
+    if (p.do_apply) grid_barrier(p.ctrl, abort_flag, false);
   }
   if (C::G > 1 && wc.f1 > wc.f0) {
     // cross-head blocks of the packed S operand are never written by a head: they must read as zero

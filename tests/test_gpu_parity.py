@@ -224,7 +224,7 @@ def test_bounded_wait_reports_timeout_and_the_context_survives(la):
     ws = la.new_workspace(q)
     good = la.linattn_state(k, v, workspace=ws).clone()
     ctrl = ws[:4096].view(torch.int32)
-    ctrl[16] = 0x4000           # arrival count of the barrier word: never equals grid - 1 again
+    ctrl[16] = 0x4000           # arrival count of the barrier word: the arrivals no longer carry into the generation
     la.linattn_state(k, v, workspace=ws)
     assert la.workspace_status(ws) == -6
     la.load_library().linattn_workspace_init(ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
