@@ -265,3 +265,43 @@ def test_work_split_with_many_units(la, orc, shape):
     ref = orc.block_masked(q, ki, vi, EPS, half)
     check("bf16", to_f64(torch.cat(outs, dim=1)), ref, f"two steps {shape}")
     assert la.workspace_status(cache.workspace) == 0
+
+
+def _random_shapes(count, seed):
+    rng = np.random.default_rng(seed)
+    shapes = []
+    while len(shapes) < count:
+        d = int(rng.choice([32, 64, 112, 128]))
+        B, H = int(rng.integers(1, 5)), int(rng.integers(1, 41))
+        N = int(rng.integers(1, 3001))
+        if B * H * N <= 150_000:
+            shapes.append((B, N, H, d))
+    return shapes
+
+
+@pytest.mark.parametrize("shape", _random_shapes(16, 20250), ids=lambda s: "B%d_N%d_H%d_d%d" % s)
+def test_seeded_random_shapes(la, orc, shape):
+    """Shapes nobody picked by hand: forward against the oracle, the state of small-integer inputs bit for bit,
+    and the same tokens as two cached steps of unequal length."""
+    import torch
+
+    B, N, H, d = shape
+    q, k, v = gen(B, N, H, d, 2400 + N, "bf16")
+    qd = to_dev(q)
+    check("bf16", to_f64(la.linattn_forward(qd, to_dev(k), to_dev(v), EPS)), orc.forward(q, k, v, EPS), f"forward {shape}")
+    ki = synth.smallint((B, N, H, d), 2401, 2, 2)
+    vi = synth.smallint((B, N, H, d), 2401, 3, 2)
+    S, z = orc.state(ki, vi)
+    got = to_f64(la.linattn_state(to_dev(ki), to_dev(vi)))
+    assert np.array_equal(got[..., :d, :].swapaxes(-1, -2), S) and np.array_equal(got[..., d, :], z)
+    cut = max(1, N // 3)
+    cache = la.BlockLinCache(B, H, d, torch.bfloat16, "cuda", max_T_b=max(cut, N - cut), eps=EPS)
+    outs = [cache.step(to_dev(np.ascontiguousarray(q[:, sl])), to_dev(np.ascontiguousarray(ki[:, sl])),
+                       to_dev(np.ascontiguousarray(vi[:, sl]))) for sl in (slice(0, cut), slice(cut, N)) if sl.stop > sl.start]
+    got = to_f64(cache.state)
+    assert np.array_equal(got[..., :d, :].swapaxes(-1, -2), S) and np.array_equal(got[..., d, :], z)
+    # the second step's rows see everything: they equal the tail of the bidirectional result on the same inputs
+    if N > cut:
+        full = la.linattn_forward(qd, to_dev(ki), to_dev(vi), EPS)
+        check("bf16", to_f64(outs[-1]), to_f64(full[:, cut:]).copy(), f"second step vs forward {shape}")
+    assert la.workspace_status(cache.workspace) == 0
