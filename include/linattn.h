@@ -227,13 +227,16 @@ LINATTN_API int blocklin_peek(blocklin_cache* cache, int64_t T_b, const void* q_
                   void* o_blk, void* stream);
 
 /* n_blocks consecutive blocks of T_b tokens in one call over [B, n_blocks*T_b, H, d] tensors; result and final
- * cache are those of n_blocks calls of blocklin_step.  q and o may both be NULL.
- * If the cache was created over a workspace of at least blocklin_prefill_workspace_bytes(desc, n_blocks, T_b)
- * bytes (and the batch stride is the dense one, or B = 1), all blocks are processed together: one state pass
- * gives every block's own state, a prefix sum over the blocks gives the cache after each block, one apply pass
- * reads every block against its prefix.  The sums are then associated differently than in n_blocks single steps,
- * so the two agree to fp32 rounding of the state, not bit for bit.  With a smaller workspace the blocks are
+ * cache are those of n_blocks calls of blocklin_step, bit for bit.  q and o may both be NULL.
+ *
+ * After blocklin_cache_joint_prefill(cache, 1), and if the cache was created over a workspace of at least
+ * blocklin_prefill_workspace_bytes(desc, n_blocks, T_b) bytes (and the batch stride is the dense one, or B = 1),
+ * all blocks are processed together instead: one state pass gives every block's own state, a prefix sum over
+ * the blocks gives the cache after each block, one apply pass reads every block against its prefix.  The sums
+ * are then associated differently than in n_blocks single steps, so the two agree to fp32 rounding of the
+ * state, not bit for bit: that is why it has to be asked for.  Where the conditions do not hold the blocks are
  * stepped one by one. */
+LINATTN_API int blocklin_cache_joint_prefill(blocklin_cache* cache, int enable);
 LINATTN_API int blocklin_prefill_workspace_bytes(const linattn_desc* desc, int64_t n_blocks, int64_t T_b,
                                                  size_t* workspace_bytes);
 LINATTN_API int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,

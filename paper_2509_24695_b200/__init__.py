@@ -93,6 +93,7 @@ def load_library(path: str | None = None):
         "blocklin_step_rope": ([vp, i64, vp, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_prefill": ([vp, i64, i64, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_prefill_workspace_bytes": ([dp, i64, i64, szp], ctypes.c_int),
+        "blocklin_cache_joint_prefill": ([vp, ctypes.c_int], ctypes.c_int),
         "blocklin_cache_info": ([vp, ctypes.POINTER(i64), ctypes.POINTER(i64), szp], ctypes.c_int),
         "blocklin_cache_destroy": ([vp], ctypes.c_int),
         "tconv_cache_bytes": ([ctypes.POINTER(_ConvDesc), szp], ctypes.c_int),
@@ -366,6 +367,8 @@ class BlockLinCache:
         _check(self._lib.blocklin_cache_init(ctypes.byref(self._handle), ctypes.byref(self._desc), eps,
                                              _ptr(self.state), sb.value, _ptr(self.workspace), nbytes,
                                              _stream(self.state)), "blocklin_cache_init")
+        if prefill_blocks > 1:
+            _check(self._lib.blocklin_cache_joint_prefill(self._handle, 1), "blocklin_cache_joint_prefill")
 
     def reset(self):
         _check(self._lib.blocklin_cache_reset(self._handle, _stream(self.state)), "blocklin_cache_reset")

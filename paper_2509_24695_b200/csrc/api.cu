@@ -166,6 +166,7 @@ struct blocklin_cache {
   size_t workspace_bytes;
   long long blocks_seen;
   long long tokens_seen;
+  int joint_prefill;   // blocklin_prefill may take all blocks together (asked for: it changes the low bits)
 };
 
 // One block: commit (cache += (S_blk, z_blk)), then read (the block's queries see the updated cache).
@@ -446,6 +447,7 @@ int blocklin_cache_init(blocklin_cache** out, const linattn_desc* desc, float ep
   c->workspace_bytes = workspace_bytes;
   c->blocks_seen = 0;
   c->tokens_seen = 0;
+  c->joint_prefill = 0;
   cudaError_t e = cudaMemsetAsync(dev_state, 0, need_state, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(dev_workspace, 0, LINATTN_WORKSPACE_CTRL_BYTES, (cudaStream_t)stream);
   if (e != cudaSuccess) {
@@ -535,7 +537,8 @@ int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const
   pv.N = T_b;
   pv.sb = T_b * p.sn;
   const bool batch_dense = p.B == 1 || p.sb == n_blocks * T_b * p.sn;
-  if (n_blocks > 1 && batch_dense && (long long)pv.B * pv.H <= 65535 && (p.state_elems() * p.H) % 4 == 0 &&
+  if (cache->joint_prefill && n_blocks > 1 && batch_dense && (long long)pv.B * pv.H <= 65535 &&
+      (p.state_elems() * p.H) % 4 == 0 &&
       cache->workspace_bytes >= workspace_need(pv)) {
     cudaStream_t s = (cudaStream_t)stream;
     float* blk = reinterpret_cast<float*>(static_cast<char*>(cache->workspace) + state_slot_offset(pv));
@@ -572,6 +575,12 @@ int blocklin_prefill_workspace_bytes(const linattn_desc* desc, int64_t n_blocks,
   pv.B = p.B * (int)n_blocks;
   const size_t steps = workspace_need(p), all = workspace_need(pv);
   *workspace_bytes = all > steps ? all : steps;
+  return LINATTN_OK;
+}
+
+int blocklin_cache_joint_prefill(blocklin_cache* cache, int enable) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  cache->joint_prefill = enable ? 1 : 0;
   return LINATTN_OK;
 }
 

@@ -190,7 +190,10 @@ struct FusedParams {
   long long N;             // tokens (bound of the rotary table)
 };
 
-constexpr int kZParts = 8 * 128;  // rotary variant: floats a partial record carries for z (per ReLU warp, per feature)
+// rotary variant: floats a partial record carries for z: per warp that sums plain phi(k) (the eight ReLU warps, and
+// the four epilogue warps, which take a share of the second K box in the state pass), per feature
+constexpr int kZSlots = 12;
+constexpr int kZParts = kZSlots * 128;
 
 // TMA coordinates (feature, head) of 64-element box `box` (0/1) of head group hg
 template <int D>
@@ -372,23 +375,30 @@ __device__ __forceinline__ void reduce_elements(const FusedParams& p, int first,
     if (ROPE && zpart[k]) {
       // rotary variant: z comes from the plain phi(k) sums that the ReLU warps of every segment left
       // behind the record (per warp, per feature): per warp slot the records in their fixed order, then the
-      // eight slots as a balanced tree (the association reduce_image's shuffles give)
+      // slots as a balanced tree over sixteen, the missing ones zero (the association reduce_image's shuffles give)
       const int e = idx % E4;
       const float4* zp = reinterpret_cast<const float4*>(p.partials) + E4 + (e - D * D / 4);
       // (one slot after the other: this form only runs when the operand images are not in use, and the
       // rotary kernel has no registers to spare)
-      float4 acc[8];
-#pragma unroll
-      for (int w = 0; w < 8; ++w) {
-        acc[w] = make_float4(0.f, 0.f, 0.f, 0.f);
+      const bool upper = e - D * D / 4 >= 16;   // features 64..: the epilogue warps' slots hold a share too
+      // (computed depth first, a few registers at a time: this form only runs when the operand images are not in
+      // use, and the rotary kernel has no registers to spare)
+      auto slot = [&](int w) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (w < 8 || (w < kZSlots && upper)) {
 #pragma unroll 2
-        for (int kk = 0; kk < nrec[k]; ++kk) add4(acc[w], __ldcg(zp + (size_t)record_of(k, kk) * REC4 + w * 32));
-      }
-#pragma unroll
-      for (int st = 1; st < 8; st *= 2)
-#pragma unroll
-        for (int w = 0; w < 8; w += 2 * st) add4(acc[w], acc[w + st]);
-      add4(sum[k], acc[0]);
+          for (int kk = 0; kk < nrec[k]; ++kk) add4(a, __ldcg(zp + (size_t)record_of(k, kk) * REC4 + w * 32));
+        }
+        return a;
+      };
+      auto pair = [&](int w) { float4 a = slot(w); add4(a, slot(w + 1)); return a; };
+      auto quad = [&](int w) { float4 a = pair(w); add4(a, pair(w + 2)); return a; };
+      float4 tree = quad(0);
+      add4(tree, quad(4));
+      float4 high = quad(8);
+      add4(high, quad(12));
+      add4(tree, high);
+      add4(sum[k], tree);
     }
     state4[idx] = sum[k];
   }
@@ -492,33 +502,36 @@ __device__ __forceinline__ void reduce_image_chunks(const FusedParams& p, int u,
   }
 }
 
-// Rotary variant: z of unit u from the plain phi(k) sums that the ReLU warps of every segment left behind the
-// record, [8 warp slots][128 features].  Thread (float4 hc of z, slot w) adds its slot over the records in their
-// fixed order (all loads in flight together), shuffles add the eight slots as a balanced tree, lane w = 0 adds
-// the old z when accumulating; two neighbouring float4 make the 32-byte chunk of the operand image.
+// Rotary variant: z of unit u from the plain phi(k) sums that the warps of every segment left behind the record,
+// [12 warp slots][128 features] (the epilogue warps' slots 8..11 only for features 64..).  Thread (float4 hc of z,
+// slot w of 16) adds its slot over the records in their fixed order (all loads in flight together; slots that
+// do not exist count as zero), shuffles add the sixteen as a balanced tree, lane w = 0 adds the old z when
+// accumulating; two neighbouring float4 make the 32-byte chunk of the operand image.
 template <int D>
 __device__ __forceinline__ void reduce_image_zrow(const FusedParams& p, int u, int ncol, int r_lo, int nrec) {
   using C = Cfg<D>;
   constexpr int E4 = (D + 1) * D / 4, REC4 = E4 + kZParts / 4, Z4 = D / 4, NR = 6;
-  static_assert((8 * Z4) % 32 == 0 && Z4 % 2 == 0, "whole warps take part in the shuffles");
+  static_assert((16 * Z4) % 32 == 0 && Z4 % 2 == 0, "whole warps take part in the shuffles");
   const int t = (int)threadIdx.x;
-  if (t >= 8 * Z4) return;
-  const int hc = t >> 3, w = t & 7;
+  if (t >= 16 * Z4) return;
+  const int hc = t >> 4, w = t & 15;
   const Sched& s = p.sa;
   auto record_of = [&](int kk) { return kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u; };
   const float4* zp = reinterpret_cast<const float4*>(p.partials) + E4 + w * 32 + hc;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int k0 = 0; k0 < nrec; k0 += NR) {
-    float4 v[NR];
+  if (w < 8 || (w < kZSlots && hc >= 16)) {
+    for (int k0 = 0; k0 < nrec; k0 += NR) {
+      float4 v[NR];
 #pragma unroll
-    for (int r = 0; r < NR; ++r)
-      if (k0 + r < nrec) v[r] = __ldcg(zp + (size_t)record_of(k0 + r) * REC4);
+      for (int r = 0; r < NR; ++r)
+        if (k0 + r < nrec) v[r] = __ldcg(zp + (size_t)record_of(k0 + r) * REC4);
 #pragma unroll
-    for (int r = 0; r < NR; ++r)
-      if (k0 + r < nrec) add4(acc, v[r]);
+      for (int r = 0; r < NR; ++r)
+        if (k0 + r < nrec) add4(acc, v[r]);
+    }
   }
 #pragma unroll
-  for (int st = 1; st < 8; st *= 2) {
+  for (int st = 1; st < 16; st *= 2) {
     float4 o;
     o.x = __shfl_xor_sync(0xffffffffu, acc.x, st); o.y = __shfl_xor_sync(0xffffffffu, acc.y, st);
     o.z = __shfl_xor_sync(0xffffffffu, acc.z, st); o.w = __shfl_xor_sync(0xffffffffu, acc.w, st);
@@ -528,8 +541,8 @@ __device__ __forceinline__ void reduce_image_zrow(const FusedParams& p, int u, i
   float4 sum = p.accumulate ? __ldcg(reinterpret_cast<const float4*>(p.state_base) + e4) : make_float4(0.f, 0.f, 0.f, 0.f);
   add4(sum, acc);
   float4 up;   // the upper half of this chunk, from the lane that holds float4 hc + 1
-  up.x = __shfl_xor_sync(0xffffffffu, sum.x, 8); up.y = __shfl_xor_sync(0xffffffffu, sum.y, 8);
-  up.z = __shfl_xor_sync(0xffffffffu, sum.z, 8); up.w = __shfl_xor_sync(0xffffffffu, sum.w, 8);
+  up.x = __shfl_xor_sync(0xffffffffu, sum.x, 16); up.y = __shfl_xor_sync(0xffffffffu, sum.y, 16);
+  up.z = __shfl_xor_sync(0xffffffffu, sum.z, 16); up.w = __shfl_xor_sync(0xffffffffu, sum.w, 16);
   if (w != 0) return;
   reinterpret_cast<float4*>(p.state)[e4] = sum;
   if (hc & 1) return;
@@ -673,7 +686,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 
   if (threadIdx.x == 0) {
     if (blockIdx.x == 0 && p.do_state) grid_barrier_preset(p.ctrl);   // for the first grid barrier
-    for (int s = 0; s < NSA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_ready[s], R::RELU_THREADS); mbar_init(&a_empty[s], 1); }
+    for (int s = 0; s < NSA; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_ready[s], R::RELU_THREADS + (ROPE ? 128 : 0)); mbar_init(&a_empty[s], 1); }
     mbar_init(a_tfull, 1);
     mbar_init(a_tempty, 128);
     mbar_init(a_done, 1);
@@ -790,13 +803,16 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     for (int e = 0; e < 8; ++e) zacc[e] = make_float2(0.f, 0.f);
     // The rotations of a row do not depend on K: they are fetched one stage ahead, each register reloaded
     // for the next stage right after its use, so that their latency is off the stage's critical path.
-    uint4 tab0[kTileState / 32], tab1[kTileState / 32];
+    // Of the second K box these warps take the first 32 token rows of a stage; the epilogue warps, idle until the
+    // segment's accumulators are complete, take the other 32 (this role is what the pass waits for).
+    uint4 tab0[kTileState / 32], tab1[1];
     auto fetch_rot = [&](int tile, int i) {
       const long long n = (long long)tile * kTileState + row0 + 32 * i;
-      tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
+      tab0[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
+      if (i == 0) tab1[0] = tab0[i];
       if (n < p.N) {
         tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
-        if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
+        if (i == 0 && box1_live) tab1[0] = __ldg(p.rope + n * (D / 8) + 8 + lc);
       }
     };
     if (ROPE) {
@@ -822,12 +838,12 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 #pragma unroll
           for (int e = 0; e < 4; ++e) zacc[e] = add2(zacc[e], f[e]);
           *c0 = rotate_pack8(f, tab0[i]);
-          if (box1_live) {
-            uint4* c1 = reinterpret_cast<uint4*>(p0 + kBox + i * 32 * kRowBytes);
+          if (i == 0 && box1_live) {
+            uint4* c1 = reinterpret_cast<uint4*>(p0 + kBox);
             unpack_relu8(*c1, f);
 #pragma unroll
             for (int e = 0; e < 4; ++e) zacc[4 + e] = add2(zacc[4 + e], f[e]);
-            *c1 = rotate_pack8(f, tab1[i]);
+            *c1 = rotate_pack8(f, tab1[0]);
           }
           if (!tn.done()) fetch_rot(tn.tile(), i);
         }
@@ -875,7 +891,67 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     const int i = wq * 32 + lane;           // accumulator lane = key feature within the group
     const int g = i / D, il = i % D;        // head within the group, feature within the head
     uint32_t seg = 0;
-    for (TileWalk t(wa); !t.done(); t.next()) {
+    // rotary variant: token rows 32..63 of the second K box of every stage (see the ReLU role); thread te owns
+    // the 16-byte column position pch of rows 32 + row0h + 16 j, which holds logical chunk lch in all of them
+    const int te = threadIdx.x - R::EPI_THREAD0;
+    const int row0h = te >> 3, pch = te & 7, lch = pch ^ (row0h & 7);
+    const bool h_live = 64 + lch * 8 < C::FEAT;
+    float2 zh[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) zh[e] = make_float2(0.f, 0.f);
+    uint4 tabh[2];
+    auto fetch_roth = [&](int tile, int j) {
+      const long long n = (long long)tile * kTileState + 32 + row0h + 16 * j;
+      tabh[j] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
+      if (h_live && n < p.N) tabh[j] = __ldg(p.rope + n * (D / 8) + 8 + lch);
+    };
+    if (ROPE) {
+      TileWalk t0(wa);
+      if (!t0.done()) { fetch_roth(t0.tile(), 0); fetch_roth(t0.tile(), 1); }
+    }
+    uint32_t it = 0;
+    for (TileWalk t(wa); !t.done(); t.next(), ++it) {
+      if (ROPE) {
+        const int s = it % NSA;
+        TileWalk tn = t;
+        tn.next();
+        if (!__all_sync(0xffffffffu, mbar_wait(&a_full[s], (it / NSA) & 1, abort_flag))) break;  // leave as a whole warp
+        uint8_t* p1 = smem + s * STAGE + C::KOFF + kBox + (32 + row0h) * kRowBytes + pch * 16;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          if (h_live) {
+            float2 f[4];
+            uint4* c1 = reinterpret_cast<uint4*>(p1 + j * 16 * kRowBytes);
+            unpack_relu8(*c1, f);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) zh[e] = add2(zh[e], f[e]);
+            *c1 = rotate_pack8(f, tabh[j]);
+          }
+          if (!tn.done()) fetch_roth(tn.tile(), j);
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(&a_ready[s]);
+        if (t.seg_last()) {
+          // this warp's share of the segment's z: the four lanes that share a chunk add up in a fixed order
+          const int rq = (te >> 3) & 3;
+          float tot[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) tot[e] = 0.f;
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) {
+            const int src = (rr << 3) | (lch ^ ((4 * ((te >> 5) & 1) + rr) & 7));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) tot[e] += __shfl_sync(0xffffffffu, (e & 1) ? zh[e >> 1].y : zh[e >> 1].x, src);
+          }
+          if (rq == 0 && h_live) {
+            float* zp = p.partials + (size_t)t.record() * (C::G * (D + 1) * D + kZParts) + C::G * (D + 1) * D + (8 + (te >> 5)) * 128;
+            *reinterpret_cast<float4*>(zp + 64 + 8 * lch) = make_float4(tot[0], tot[1], tot[2], tot[3]);
+            *reinterpret_cast<float4*>(zp + 64 + 8 * lch + 4) = make_float4(tot[4], tot[5], tot[6], tot[7]);
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) zh[e] = make_float2(0.f, 0.f);
+        }
+      }
       if (!t.seg_last()) continue;
       bool ok = mbar_wait(a_tfull, seg & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
