@@ -409,6 +409,23 @@ def extras(torch, la, synth, dev, peak):
                        "cache_bytes_at_first_and_last_step": [cache.info()["state_bytes"]] * 2,
                        "l2": "block set of %.0f MB cycled over 3 copies" % (step_bytes / 1e6)}
         del graph
+        if w.name == synth.STREAM720.name:
+            # the same steps with the rotary factors of Eq. 2 (blocklin_step_rope); the block's rows of a 3D table
+            cos, sin = synth.rope_table(3, 45, 80, w.d)
+            table = la.rope_pack(torch.from_numpy(cos).to(dev), torch.from_numpy(sin).to(dev))
+            for i in range(3):
+                cache.step_rope(*blocks[i % 3], table, out=ob)
+            tp = ctypes.c_void_p(table.data_ptr())
+
+            def rope_steps(i):
+                qp, kp, vp_ = ptrs[i % 3]
+                if lib.blocklin_step_rope(cache._handle, w.T_b, qp, kp, vp_, op, tp, stream) != 0:
+                    raise RuntimeError("blocklin_step_rope failed")
+
+            us_rope = time_loop(torch, rope_steps, n_steps) / n_steps * 1e3
+            res[w.name]["step_latency_us_rope"] = us_rope
+            res[w.name]["frac_of_peak_rope"] = step_bytes / (us_rope * 1e-6) / 1e9 / peak
+            del table
         cache.close()
         del blocks, ob
     # the 7 context blocks of the autoregressive 480p layer in one prefill call: block by block, and all together
