@@ -195,3 +195,38 @@ def test_denoise_loop_reads_without_committing(la, orc, dtype, d):
         orc.block_step((S, z), q, k, v, EPS, want_o=False)
         assert_state_close(to_f64(cache.state), S, z, 1e-5, f"cache after block {blk}")
     assert cache.info()["blocks_seen"] == M
+
+
+def test_steps_replay_from_a_cuda_graph(la):
+    """A run of cached steps captured into a CUDA graph and replayed gives the bits of the same steps launched one
+    by one (every call only enqueues work on the stream it is given; nothing is allocated or synchronised)."""
+    import ctypes
+
+    import torch
+
+    B, H, d, T_b, M = 1, 4, 112, 520, 3
+    q, k, v = (to_dev(x) for x in gen(B, T_b * M, H, d, 3300, "bf16"))
+    blocks = [tuple(t[:, i * T_b:(i + 1) * T_b].contiguous() for t in (q, k, v)) for i in range(M)]
+    cache = la.BlockLinCache(B, H, d, torch.bfloat16, "cuda", max_T_b=T_b, eps=EPS)
+    eager = [cache.step(*blk) for blk in blocks]          # also the warm-up a capture needs
+    final = cache.state.clone()
+    outs = [torch.empty_like(o) for o in eager]
+    lib = la.load_library()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        cache.reset()
+        with torch.cuda.graph(graph, stream=side):
+            handle = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+            for (qb, kb, vb), ob in zip(blocks, outs):
+                assert lib.blocklin_step(cache._handle, T_b, qb.data_ptr(), kb.data_ptr(), vb.data_ptr(), ob.data_ptr(),
+                                         handle) == 0
+        for _ in range(2):                                  # replay twice: the second one starts from a reset cache too
+            cache.reset()
+            graph.replay()
+            side.synchronize()
+            assert all(torch.equal(a, b) for a, b in zip(outs, eager))
+            assert torch.equal(cache.state, final)
+    torch.cuda.current_stream().wait_stream(side)
+    assert la.workspace_status(cache.workspace) == 0
