@@ -71,3 +71,21 @@ def sample_rows(N, count, seed, tile=128):
     fixed = [r for r in fixed if 0 <= r < N]
     rnd = rng.integers(0, N, size=max(0, count - len(fixed)))
     return np.unique(np.concatenate([np.array(fixed, dtype=np.int64), rnd.astype(np.int64)]))
+
+
+def read_golden(name):
+    """Sections of a text fixture under tests/golden/: {'section': float64 array}, comment lines skipped."""
+    import os
+
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)
+    out, key = {}, None
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("["):
+            key = line.strip("[]")
+            out[key] = []
+        else:
+            out[key].append([float(x) for x in line.split()])
+    return {k: np.array(v, dtype=np.float64) for k, v in out.items()}

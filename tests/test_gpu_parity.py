@@ -305,3 +305,20 @@ def test_seeded_random_shapes(la, orc, shape):
         full = la.linattn_forward(qd, to_dev(ki), to_dev(vi), EPS)
         check("bf16", to_f64(outs[-1]), to_f64(full[:, cut:]).copy(), f"second step vs forward {shape}")
     assert la.workspace_status(cache.workspace) == 0
+
+
+def test_hand_worked_example_on_the_gpu(la):
+    """The hand-worked d = 2 example of tests/golden/ through the library itself (fp32 I/O path)."""
+    import torch
+    from parity_util import read_golden
+
+    g = read_golden("eq2_eq3_hand_worked_d2.txt")
+    q, k, v = (torch.from_numpy(g[n].reshape(1, 3, 1, 2).astype(np.float32)).cuda() for n in ("q", "k", "v"))
+    st = to_f64(la.linattn_state(k, v))
+    assert np.array_equal(st[0, 0, :2].T, g["S"]) and np.array_equal(st[0, 0, 2], g["z"][0])
+    assert np.allclose(to_f64(la.linattn_forward(q, k, v, 0.0))[0, :, 0], g["o_bidirectional_eps0"], rtol=2e-7, atol=0)
+    assert np.allclose(to_f64(la.linattn_forward(q, k, v, 0.5))[0, :, 0], g["o_bidirectional_eps_half"], rtol=2e-7, atol=0)
+    cache = la.BlockLinCache(1, 1, 2, torch.float32, "cuda", max_T_b=2, eps=0.0)
+    o12 = cache.step(q[:, :2].contiguous(), k[:, :2].contiguous(), v[:, :2].contiguous())
+    o3 = cache.step(q[:, 2:].contiguous(), k[:, 2:].contiguous(), v[:, 2:].contiguous())
+    assert np.allclose(to_f64(torch.cat([o12, o3], dim=1))[0, :, 0], g["o_blocks_12_3_eps0"], rtol=2e-7, atol=0)

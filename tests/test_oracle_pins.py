@@ -57,6 +57,28 @@ def pin_hand_worked_example(o):
     assert np.array_equal(cache[0][0, 0], [[1.0, 0.0], [2.0, 2.0]]) and np.array_equal(cache[1][0, 0], [1.0, 3.0])
 
 
+def pin_golden_hand_worked_d2(o):
+    """tests/golden/eq2_eq3_hand_worked_d2.txt: Eq. 2 and Eq. 3 worked by hand (derivation in the file)."""
+    from parity_util import read_golden
+
+    g = read_golden("eq2_eq3_hand_worked_d2.txt")
+    q, k, v = (g[n].reshape(1, 3, 1, 2) for n in ("q", "k", "v"))
+    S, z = o.state(k, v)
+    assert np.array_equal(S[0, 0], g["S"]) and np.array_equal(z[0, 0], g["z"][0])
+    for fn in (o.forward, o.quadratic):
+        assert np.allclose(fn(q, k, v, 0.0)[0, :, 0], g["o_bidirectional_eps0"], rtol=0, atol=2e-16)
+        assert np.allclose(fn(q, k, v, 0.5)[0, :, 0], g["o_bidirectional_eps_half"], rtol=0, atol=2e-16)
+    for out in (o.quadratic(q, k, v, 0.0, 1), o.block_masked(q, k, v, 0.0, 1)):
+        assert np.allclose(out[0, :, 0], g["o_blocks_of_one_eps0"], rtol=0, atol=2e-16)
+    for out in (o.quadratic(q, k, v, 0.0, 2), o.block_masked(q, k, v, 0.0, 2)):
+        assert np.allclose(out[0, :, 0], g["o_blocks_12_3_eps0"], rtol=0, atol=2e-16)
+    cache = o.new_cache(1, 1, 2)
+    o12 = o.block_step(cache, q[:, :2], k[:, :2], v[:, :2], 0.0)
+    o3 = o.block_step(cache, q[:, 2:], k[:, 2:], v[:, 2:], 0.0)
+    assert np.allclose(np.concatenate([o12, o3], axis=1)[0, :, 0], g["o_blocks_12_3_eps0"], rtol=0, atol=2e-16)
+    assert np.array_equal(cache[0][0, 0], g["S"]) and np.array_equal(cache[1][0, 0], g["z"][0])
+
+
 def pin_exact_rational(o):
     """Small-integer inputs: the definition evaluated in exact rational arithmetic."""
     N, d = 5, 3
@@ -345,7 +367,7 @@ def pin_rope_linear_equals_quadratic_and_shift(o):
     assert np.array_equal(full[1:, :, 1:], part)
 
 
-PINS = [pin_hand_worked_example, pin_exact_rational, pin_linear_equals_quadratic, pin_bf16_decode_and_tiny_config,
+PINS = [pin_hand_worked_example, pin_golden_hand_worked_d2, pin_exact_rational, pin_linear_equals_quadratic, pin_bf16_decode_and_tiny_config,
         pin_constant_v, pin_single_token, pin_one_hot_is_segment_mean, pin_invariances, pin_sign, pin_convexity,
         pin_block_forms_agree, pin_cache_size_constant, pin_strides_and_rows, pin_rope_closed_form_d2,
         pin_rope_reduces_to_plain, pin_rope_linear_equals_quadratic_and_shift]

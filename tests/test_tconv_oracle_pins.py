@@ -126,7 +126,27 @@ def pin_bf16_bits_and_small_integers(o):
     assert np.array_equal(y[0, :, 0, 1], [-1 - 20 + 0, 0 - 2 + 0 - 800, -4 + 0 - 80])
 
 
-PINS = [pin_bidirectional_is_library_correlation, pin_blocks_of_one_frame_are_a_causal_filter, pin_impulse_responses,
+def pin_golden_hand_worked(o):
+    """tests/golden/tconv_hand_worked.txt: four frames, two channels, worked by hand (derivation in the file)."""
+    import sys
+
+    sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+    from parity_util import read_golden
+
+    g = read_golden("tconv_hand_worked.txt")
+    x = g["x"].reshape(1, 4, 1, 2)
+    assert np.array_equal(o.tconv_bidirectional(x, g["w"])[0, :, 0], g["y_bidirectional"])
+    assert np.array_equal(o.tconv_block_masked(x, g["w"], 2)[0, :, 0], g["y_blocks_of_two"])
+    f = o.new_cache(1, 1, 2)
+    ys = []
+    for t0 in (0, 2):
+        y, f = o.tconv_block_step(x[:, t0:t0 + 2], g["w"], f)
+        ys.append(y)
+    assert np.array_equal(np.concatenate(ys, axis=1)[0, :, 0], g["y_blocks_of_two"])
+    assert np.array_equal(f[0, 0], g["cache_after"][0])
+
+
+PINS = [pin_golden_hand_worked, pin_bidirectional_is_library_correlation, pin_blocks_of_one_frame_are_a_causal_filter, pin_impulse_responses,
         pin_zero_taps_is_identity_and_centre_tap_scales, pin_causality_across_blocks, pin_stepping_equals_one_shot,
         pin_bf16_bits_and_small_integers]
 
