@@ -215,3 +215,21 @@ def test_full_size_block_causal(la, wl):
     assert torch.equal(cache.frame, xd[:, -1])
     cache.reset()
     assert torch.equal(cache.prefill(xd, wd, wl.T // wl.T_b), y)
+
+
+def test_hand_worked_example_on_the_gpu(la):
+    """The hand-worked example of tests/golden/tconv_hand_worked.txt through the library (fp32 path; its two channels
+    repeated to the four the 16-byte pieces need, at three positions)."""
+    import torch
+    from parity_util import read_golden
+
+    g = read_golden("tconv_hand_worked.txt")
+    tile = lambda a: np.tile(a, (1, 2)).astype(np.float32)            # [T or 3, 2] -> [.., 4]
+    x = torch.from_numpy(np.repeat(tile(g["x"])[None, :, None, :], 3, axis=2)).cuda().contiguous()   # [1, 4, 3, 4]
+    w = torch.from_numpy(tile(g["w"])).cuda().contiguous()
+    y = to_f64(la.tconv_forward(x, w))
+    assert all(np.array_equal(y[0, :, p], tile(g["y_bidirectional"])) for p in range(3))
+    cache = la.TConvCache(1, 3, 4, torch.float32, "cuda")
+    yb = to_f64(torch.cat([cache.step(x[:, t0:t0 + 2], w) for t0 in (0, 2)], dim=1))
+    assert all(np.array_equal(yb[0, :, p], tile(g["y_blocks_of_two"])) for p in range(3))
+    assert np.array_equal(to_f64(cache.frame)[0, 0], tile(g["cache_after"])[0])
