@@ -11,13 +11,17 @@
 //                operands; the contraction index is the token.  The "ones" column makes z fall out of
 //                the same MMA as one more accumulator column.  Work is split over tokens across the
 //                grid (split-N); every CTA writes one fp32 partial record per unit segment it covered.
-//   reduce       after a grid barrier every CTA sums a slice of the state over the partial records in
-//                a fixed order (deterministic), optionally on top of the existing state: the cache
-//                update of Eq. 3.  A second grid barrier publishes the state.
+//   reduce       after a grid barrier the state is summed over the partial records in a fixed order
+//                (deterministic), optionally on top of the existing state: the cache update of Eq. 3.
+//                Either every CTA sums a slice of the whole state, or (one-head units, fused launch) the
+//                CTAs of a unit share its reduce and also leave the unit's apply operand (S as bf16
+//                hi + lo, z as one more row, in the shared-memory layout) in a per-unit image.  A second
+//                grid barrier publishes state and images.
 //   apply pass   o_n = phi(q_n) S / (phi(q_n).z + eps).  A = phi(Q) tile (K-major), B = S split into
 //                bf16 hi + lo parts (two MMAs per K step, so S keeps ~16 mantissa bits), with z as an
-//                extra row of B so the denominator is one more accumulator column.  The epilogue
-//                divides, rounds to bf16 and a dedicated warp TMA-stores the tile.
+//                extra row of B so the denominator is one more accumulator column.  B comes into shared
+//                memory once per unit segment: one bulk copy of the unit's image, or built from the fp32
+//                state.  The epilogue divides, rounds to bf16 and a dedicated warp TMA-stores the tile.
 //
 // The first Q tiles of the apply pass are fetched before the grid barriers (Q does not depend on the
 // state), so HBM stays busy while the partials are reduced.
