@@ -49,7 +49,7 @@ def parse():
 
 
 def workload_of(name):
-    from paper_2509_24695_b200 import synth
+    import synth
 
     return synth.P480 if name == "480p" else synth.P720
 
@@ -143,7 +143,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    from paper_2509_24695_b200 import synth
+    import synth
     import oracle
 
     w = workload_of(args.workload)
@@ -213,7 +213,7 @@ def main():
 
     import torch
     import paper_2509_24695_b200 as la
-    from paper_2509_24695_b200 import synth
+    import synth
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -153,8 +153,11 @@ LINATTN_API int linattn_state(const linattn_desc* desc, int64_t N, const void* k
  *
  *  - Limit: the scratch the call needs (what linattn_workspace_bytes reports, minus the trailing
  *    state slot) must fit in LINATTN_STATIC_SCRATCH_BYTES (16 MiB; every GPU on which this library
- *    is used holds that much device memory until the process exits).  That covers, for example,
- *    B*H <= 20 heads of dimension 112 at any N.  Larger problems return
+ *    is used holds that much device memory until the process exits).  For bf16 inputs with
+ *    d in {32 (heads contiguous), 64, 112, 128} the need does not grow with N, and B*H <= 20 heads
+ *    of dimension 112 fit at any N.  Other shapes and fp32 inputs keep one partial state per 512
+ *    tokens (at most 64) per head, so they fit only while B*H*(d*d+d)*4*min(64, ceil(N/512)) stays
+ *    below the limit (20 fp32 heads of dimension 112: N <= 8192).  Larger problems return
  *    LINATTN_ERR_SCRATCH_LIMIT and launch nothing.
  *  - The first call on each device looks the array's device address up (one runtime call, with
  *    that device current); make that first call outside any stream capture.
@@ -165,6 +168,11 @@ LINATTN_API int linattn_state(const linattn_desc* desc, int64_t N, const void* k
 #define LINATTN_STATIC_SCRATCH_BYTES (16u << 20)
 LINATTN_API int linattn_state_static_scratch(const linattn_desc* desc, int64_t N, const void* k, const void* v,
                                              float* state, void* stream);
+
+/* linattn_workspace_status for the built-in array (its address is not the caller's to know): synchronises
+ * `stream`, then reports LINATTN_OK or LINATTN_ERR_TIMEOUT of the LAST linattn_state_static_scratch call on the
+ * current device through *status (every call clears the word before its launch).  (No counterpart in the paper.) */
+LINATTN_API int linattn_static_scratch_status(void* stream, int* status);
 
 /* The apply half of Eq. 2 alone: o_n = phi(q_n) S / (phi(q_n) . z + eps) for a given state.
  * workspace: only its control block is used (LINATTN_WORKSPACE_CTRL_BYTES suffice). */
@@ -202,7 +210,8 @@ LINATTN_API int blocklin_cache_bytes(const linattn_desc* desc, int64_t max_T_b, 
 LINATTN_API int blocklin_cache_init(blocklin_cache** out, const linattn_desc* desc, float eps, void* dev_state,
                         size_t state_bytes, void* dev_workspace, size_t workspace_bytes, void* stream);
 
-/* Forget the past: zero the state, blocks_seen = tokens_seen = 0. */
+/* Forget the past: zero the state, blocks_seen = tokens_seen = 0.  Also zeroes the control block of the cache's
+ * workspace, which clears a recorded LINATTN_ERR_TIMEOUT (see blocklin_cache_status). */
 LINATTN_API int blocklin_cache_reset(blocklin_cache* cache, void* stream);
 
 /* One block of T_b tokens ([B, T_b, H, d] with the descriptor's strides): add the block's own
@@ -215,9 +224,22 @@ LINATTN_API int blocklin_step(blocklin_cache* cache, int64_t T_b, const void* q_
  * holds (sum of RoPE(phi(k))^T v, sum of phi(k)).  rope_table_blk: the packed (cos, sin) fp16 rows of this block's
  * T_b tokens ([T_b][d/2], see linattn_forward_rope); positions simply continue from block to block, so it is
  * usually a pointer into one table of the whole stream.  A stream uses either this call or blocklin_step for
- * all of its blocks.  q_blk and o_blk are required. */
+ * all of its blocks.  o_blk and q_blk may both be NULL: absorb only. */
 LINATTN_API int blocklin_step_rope(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk,
                                    const void* v_blk, void* o_blk, const void* rope_table_blk, void* stream);
+
+/* blocklin_peek with the rotary factors: a denoising step of Algorithm 1 on the attention the model runs (Eq. 2
+ * with RoPE, Sec. 3.1).  The block's queries see the rotary cache plus the block's own rotated state; the cache is
+ * only read and blocks_seen does not change.  Same bits as blocklin_step_rope would give on the same cache.
+ * q_blk and o_blk are required. */
+LINATTN_API int blocklin_peek_rope(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk,
+                                   const void* v_blk, void* o_blk, const void* rope_table_blk, void* stream);
+
+/* blocklin_prefill with the rotary factors: n_blocks consecutive blocks of T_b tokens over [B, n_blocks*T_b, H, d]
+ * tensors, rope_table the packed rows of those n_blocks*T_b tokens; result and final cache are those of n_blocks
+ * calls of blocklin_step_rope, bit for bit (the blocks are stepped one by one).  q and o may both be NULL. */
+LINATTN_API int blocklin_prefill_rope(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,
+                                      const void* v, void* o, const void* rope_table, void* stream);
 
 /* The denoising steps of Algorithm 1 ("x0 <- G(x; t_j, KV)" for t_j > 0): the block's queries see the
  * cache plus the block's own (S_blk, z_blk), exactly as in blocklin_step, but the cache is only read:
@@ -225,6 +247,25 @@ LINATTN_API int blocklin_step_rope(blocklin_cache* cache, int64_t T_b, const voi
  * blocklin_step (with q_blk = o_blk = NULL to commit without producing outputs). */
 LINATTN_API int blocklin_peek(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
                   void* o_blk, void* stream);
+
+/* ---- a block whose tokens are spread over several GPUs ----
+ * The state of Eq. 2 and the running sums of Eq. 3 are sums over tokens, so a block (or a whole sequence) can be
+ * split by tokens over ranks: every rank reduces its own shard, ONE all-reduce (sum) of B*H*(d*d+d) floats makes
+ * the new cache on every rank, and every rank applies its own queries to it.  The library does the two local
+ * halves; the all-reduce is the caller's (NCCL through torch.distributed in the Python binding), on memory of
+ * the caller's own GPU.
+ *
+ * blocklin_shard_state: state_out (DEVICE, one state, not the cache's own memory) = this rank's share of the new
+ *   cache: the state of its T_shard tokens of the block, plus the current cache when include_cache is non-zero.
+ *   Exactly ONE rank passes include_cache = 1, so that the sum over ranks is cache + state(block).  The cache is
+ *   only read.  T_shard = 0 is allowed (state_out = the cache, or zeros).
+ * blocklin_shard_commit: the cache := state_in (the all-reduced sum; every rank passes the same values),
+ *   blocks_seen += 1, tokens_seen += block_tokens (the block's tokens over all ranks).
+ * The block's outputs are then linattn_apply(q_shard, cache state) on each rank.  With one rank and
+ * include_cache = 1 the three calls give the bits of blocklin_step. */
+LINATTN_API int blocklin_shard_state(blocklin_cache* cache, int64_t T_shard, const void* k_shard, const void* v_shard,
+                                     float* state_out, int include_cache, void* stream);
+LINATTN_API int blocklin_shard_commit(blocklin_cache* cache, const float* state_in, int64_t block_tokens, void* stream);
 
 /* n_blocks consecutive blocks of T_b tokens in one call over [B, n_blocks*T_b, H, d] tensors; result and final
  * cache are those of n_blocks calls of blocklin_step, bit for bit.  q and o may both be NULL.
@@ -245,6 +286,14 @@ LINATTN_API int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_
 /* Host-side bookkeeping; any out-param may be NULL. */
 LINATTN_API int blocklin_cache_info(const blocklin_cache* cache, int64_t* blocks_seen, int64_t* tokens_seen,
                         size_t* state_bytes);
+
+/* Device-side status of the stream's launches so far.  Launches are asynchronous, so a bounded device-side wait
+ * that ran out (Sec. 3.2's step is one cooperative launch with two grid-wide meetings) cannot be reported by the
+ * call that enqueued it: this call synchronises `stream` and reports LINATTN_OK or LINATTN_ERR_TIMEOUT through
+ * *status.  After a timeout the outputs of that launch are undefined and the workspace's barrier word is left
+ * half-counted, so every later launch on this cache would time out as well: call blocklin_cache_reset (or restore
+ * a checkpoint of the state and call linattn_workspace_init on the workspace) before going on. */
+LINATTN_API int blocklin_cache_status(const blocklin_cache* cache, void* stream, int* status);
 
 /* Frees the host handle only; device memory stays the caller's. */
 LINATTN_API int blocklin_cache_destroy(blocklin_cache* cache);

@@ -54,6 +54,7 @@ def _bind(path: str):
     lib.oracle_rope_forward.argtypes = [sp, vp, vp, vp, dp, dp, f64, dp]
     lib.oracle_rope_quadratic.argtypes = [sp, vp, vp, vp, dp, dp, f64, i64, dp]
     lib.oracle_rope_block_masked.argtypes = [sp, vp, vp, vp, dp, dp, f64, i64, dp]
+    lib.oracle_rope_block_step.argtypes = [sp, vp, vp, vp, dp, dp, f64, dp, dp, dp]
     lib.oracle_cache_bytes.argtypes = [i64, i64, i64]
     lib.oracle_cache_bytes.restype = i64
     return lib
@@ -146,6 +147,19 @@ class Oracle:
         o = np.empty((s.B, s.N, s.H, s.d)) if want_o else None
         self._lib.oracle_block_step(ctypes.byref(s), q.ctypes.data, k.ctypes.data, v.ctypes.data, eps,
                                     self._dp(S), self._dp(z), self._dp(o) if want_o else None)
+        return o
+
+    def rope_block_step(self, cache, q, k, v, cos_blk, sin_blk, eps, want_o: bool = True):
+        """``block_step`` with rotary factors: cache += (RoPE(phi(k))^T v, phi(k)) of the block, then the block's
+        queries read it.  cos_blk, sin_blk: [T_b, d//2], the table rows of the block's tokens."""
+        S, z = cache
+        s = self._shape(q, k, v)
+        cs = np.ascontiguousarray(cos_blk, dtype=np.float64)
+        sn = np.ascontiguousarray(sin_blk, dtype=np.float64)
+        assert cs.shape == sn.shape == (s.N, s.d // 2)
+        o = np.empty((s.B, s.N, s.H, s.d)) if want_o else None
+        self._lib.oracle_rope_block_step(ctypes.byref(s), q.ctypes.data, k.ctypes.data, v.ctypes.data, self._dp(cs),
+                                         self._dp(sn), eps, self._dp(S), self._dp(z), self._dp(o) if want_o else None)
         return o
 
     def cache_bytes(self, B, H, d) -> int:

@@ -304,10 +304,39 @@ void oracle_rope_quadratic(const oracle_shape* s, const void* q, const void* k, 
   }
 }
 
-/* Block-causal form with rotary factors, block by block with the cache (Eq. 3 applied to Eq. 2's right-hand
- * form): the cache holds (sum of RoPE(phi(k))^T v, sum of phi(k)); each block is added, then its queries are
- * applied (rotated for the numerator, plain for the denominator).  Token n of the sequence uses row n of the
- * tables.  o: [B,N,H,d] dense fp64. */
+/* One block of the block-causal form with rotary factors (Eq. 3's running sums applied to Eq. 2's right-hand
+ * form): the cache (S, z) of one (b, h) holds (sum of RoPE(phi(k))^T v, sum of phi(k)); the block's tokens
+ * [n0, n1) are added to it, then the block's queries are applied to it (rotated for the numerator, plain for
+ * the denominator).  Token n of the tensors uses row n of the tables.  o may be NULL (commit only). */
+static void rope_block(const oracle_shape* s, const void* q, const void* k, const void* v, const double* cs,
+                       const double* sn, int64_t b, int64_t h, int64_t n0, int64_t n1, double eps, double* S,
+                       double* z, double* plain, double* rot, double* o) {
+  const int64_t d = s->d;
+  for (int64_t n = n0; n < n1; ++n) { /* commit the block ... */
+    const int64_t base = at(s, b, n, h);
+    rope_features(s, k, base, cs, sn, n, plain, rot);
+    for (int64_t i = 0; i < d; ++i) {
+      z[i] += plain[i];
+      for (int64_t j = 0; j < d; ++j) S[i * d + j] += rot[i] * load_elem(v, s->dtype, base + j);
+    }
+  }
+  if (!o) return;
+  for (int64_t n = n0; n < n1; ++n) { /* ... then read it */
+    double* o_row = o + ((b * s->N + n) * s->H + h) * d;
+    rope_features(s, q, at(s, b, n, h), cs, sn, n, plain, rot);
+    double den = 0.0;
+    for (int64_t j = 0; j < d; ++j) o_row[j] = 0.0;
+    for (int64_t i = 0; i < d; ++i) {
+      den += plain[i] * z[i];
+      for (int64_t j = 0; j < d; ++j) o_row[j] += rot[i] * S[i * d + j];
+    }
+    den += eps;
+    for (int64_t j = 0; j < d; ++j) o_row[j] /= den;
+  }
+}
+
+/* Block-causal form with rotary factors over a whole sequence, block by block from an empty cache.
+ * o: [B,N,H,d] dense fp64. */
 void oracle_rope_block_masked(const oracle_shape* s, const void* q, const void* k, const void* v, const double* cs,
                               const double* sn, double eps, int64_t T_b, double* o) {
   const int64_t d = s->d, BH = s->B * s->H;
@@ -316,32 +345,26 @@ void oracle_rope_block_masked(const oracle_shape* s, const void* q, const void* 
     const int64_t b = u / s->H, h = u % s->H;
     double* S = (double*)calloc((size_t)(d * d + 3 * d), sizeof(double));
     double* z = S + d * d;
-    double* plain = z + d;
-    double* rot = plain + d;
     for (int64_t n0 = 0; n0 < s->N; n0 += T_b) {
       const int64_t n1 = n0 + T_b < s->N ? n0 + T_b : s->N;
-      for (int64_t n = n0; n < n1; ++n) { /* commit the block ... */
-        const int64_t base = at(s, b, n, h);
-        rope_features(s, k, base, cs, sn, n, plain, rot);
-        for (int64_t i = 0; i < d; ++i) {
-          z[i] += plain[i];
-          for (int64_t j = 0; j < d; ++j) S[i * d + j] += rot[i] * load_elem(v, s->dtype, base + j);
-        }
-      }
-      for (int64_t n = n0; n < n1; ++n) { /* ... then read it */
-        double* o_row = o + ((b * s->N + n) * s->H + h) * d;
-        rope_features(s, q, at(s, b, n, h), cs, sn, n, plain, rot);
-        double den = 0.0;
-        for (int64_t j = 0; j < d; ++j) o_row[j] = 0.0;
-        for (int64_t i = 0; i < d; ++i) {
-          den += plain[i] * z[i];
-          for (int64_t j = 0; j < d; ++j) o_row[j] += rot[i] * S[i * d + j];
-        }
-        den += eps;
-        for (int64_t j = 0; j < d; ++j) o_row[j] /= den;
-      }
+      rope_block(s, q, k, v, cs, sn, b, h, n0, n1, eps, S, z, z + d, z + 2 * d, o);
     }
     free(S);
+  }
+}
+
+/* One cached step with rotary factors on a caller-held cache: S [B,H,d,d], z [B,H,d] are updated in place
+ * (Algorithm 1's cache update), o [B,N,H,d] gets the block's outputs (NULL: commit only).  The tensors hold
+ * the block alone (N = its tokens) and cs, sn are the table rows of those tokens.  A read-only denoising step
+ * is this function run on a copy of the cache. */
+void oracle_rope_block_step(const oracle_shape* s, const void* q, const void* k, const void* v, const double* cs,
+                            const double* sn, double eps, double* S, double* z, double* o) {
+  const int64_t d = s->d, BH = s->B * s->H;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t u = 0; u < BH; ++u) {
+    double* tmp = (double*)calloc((size_t)(2 * d), sizeof(double));
+    rope_block(s, q, k, v, cs, sn, u / s->H, u % s->H, 0, s->N, eps, S + u * d * d, z + u * d, tmp, tmp + d, o);
+    free(tmp);
   }
 }
 

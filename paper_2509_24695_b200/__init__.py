@@ -18,7 +18,7 @@ import os
 
 __all__ = [
     "LinAttnError", "library_path", "load_library", "state_bytes", "workspace_bytes", "new_workspace",
-    "linattn_forward", "linattn_forward_rope", "rope_pack", "new_rope_workspace", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
+    "linattn_forward", "linattn_forward_rope", "rope_pack", "new_rope_workspace", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "static_scratch_status", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
     "tconv_forward", "TConvCache",
 ]
 
@@ -91,7 +91,13 @@ def load_library(path: str | None = None):
         "blocklin_step": ([vp, i64, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_peek": ([vp, i64, vp, vp, vp, vp, vp], ctypes.c_int),
         "blocklin_step_rope": ([vp, i64, vp, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_peek_rope": ([vp, i64, vp, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_prefill_rope": ([vp, i64, i64, vp, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_cache_status": ([vp, vp, ctypes.POINTER(ctypes.c_int)], ctypes.c_int),
+        "linattn_static_scratch_status": ([vp, ctypes.POINTER(ctypes.c_int)], ctypes.c_int),
         "blocklin_prefill": ([vp, i64, i64, vp, vp, vp, vp, vp], ctypes.c_int),
+        "blocklin_shard_state": ([vp, i64, vp, vp, vp, ctypes.c_int, vp], ctypes.c_int),
+        "blocklin_shard_commit": ([vp, vp, i64, vp], ctypes.c_int),
         "blocklin_prefill_workspace_bytes": ([dp, i64, i64, szp], ctypes.c_int),
         "blocklin_cache_joint_prefill": ([vp, ctypes.c_int], ctypes.c_int),
         "blocklin_cache_info": ([vp, ctypes.POINTER(i64), ctypes.POINTER(i64), szp], ctypes.c_int),
@@ -313,6 +319,16 @@ def linattn_state_static_scratch(k, v, out):
     return out
 
 
+def static_scratch_status(device=None) -> int:
+    """Device-side status (0 or -6) of the last ``linattn_state_static_scratch`` call on the current device."""
+    torch = _torch()
+    lib = load_library()
+    st = ctypes.c_int(0)
+    _check(lib.linattn_static_scratch_status(torch.cuda.current_stream(device).cuda_stream, ctypes.byref(st)),
+           "linattn_static_scratch_status")
+    return st.value
+
+
 def linattn_apply(q, state, eps: float = 1e-6, out=None, workspace=None):
     """Apply half of Eq. 2 for a given state."""
     torch = _torch()
@@ -362,7 +378,7 @@ class BlockLinCache:
                                                               ctypes.byref(pb)), "blocklin_prefill_workspace_bytes")
             nbytes = max(nbytes, pb.value)
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
-        self.max_T_b = max_T_b
+        self.max_T_b, self.eps = max_T_b, eps
         self._handle = ctypes.c_void_p()
         _check(self._lib.blocklin_cache_init(ctypes.byref(self._handle), ctypes.byref(self._desc), eps,
                                              _ptr(self.state), sb.value, _ptr(self.workspace), nbytes,
@@ -387,20 +403,55 @@ class BlockLinCache:
                "blocklin_step")
         return o
 
+    def _rope_args(self, q, k, v, table, out, rows):
+        torch = _torch()
+        o = None
+        if q is not None:
+            o = torch.empty_like(q) if out is None else out
+            _desc_of(q, k, v, o)
+        else:
+            _desc_of(k, v)
+        self._check_layout(k)
+        d = k.shape[3]
+        if tuple(table.shape) != (rows, d // 2, 2) or table.dtype != torch.float16 or not table.is_contiguous() \
+                or table.device != k.device:
+            raise ValueError("the rotary table must be a contiguous float16 [tokens, d//2, 2] tensor on the blocks' device")
+        return o
+
     def step_rope(self, q, k, v, rope_table_blk, out=None):
         """``step`` with rotary factors; rope_table_blk: float16 [T_b, d//2, 2] rows of the block's tokens
-        (a contiguous slice of the stream's ``rope_pack`` table)."""
-        torch = _torch()
-        o = torch.empty_like(q) if out is None else out
-        _desc_of(q, k, v, o)
-        self._check_layout(k)
-        T_b, d = k.shape[1], k.shape[3]
-        if tuple(rope_table_blk.shape) != (T_b, d // 2, 2) or rope_table_blk.dtype != torch.float16 or \
-                not rope_table_blk.is_contiguous():
-            raise ValueError("rope_table_blk must be a contiguous float16 [T_b, d//2, 2] tensor")
-        _check(self._lib.blocklin_step_rope(self._handle, T_b, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(rope_table_blk),
-                                            _stream(k)), "blocklin_step_rope")
+        (a contiguous slice of the stream's ``rope_pack`` table).  q may be None: absorb only."""
+        o = self._rope_args(q, k, v, rope_table_blk, out, k.shape[1])
+        _check(self._lib.blocklin_step_rope(self._handle, k.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                                            _ptr(rope_table_blk), _stream(k)), "blocklin_step_rope")
         return o
+
+    def peek_rope(self, q, k, v, rope_table_blk, out=None):
+        """``peek`` with rotary factors: the block against the rotary cache plus itself, nothing committed."""
+        if q is None:
+            raise ValueError("peek_rope needs queries")
+        o = self._rope_args(q, k, v, rope_table_blk, out, k.shape[1])
+        _check(self._lib.blocklin_peek_rope(self._handle, k.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                                            _ptr(rope_table_blk), _stream(k)), "blocklin_peek_rope")
+        return o
+
+    def prefill_rope(self, q, k, v, rope_table, n_blocks: int, out=None):
+        """n_blocks equal blocks with rotary factors in one call; rope_table: the rows of all their tokens."""
+        N = k.shape[1]
+        if n_blocks <= 0 or N % n_blocks:
+            raise ValueError("token count must be n_blocks * T_b")
+        o = self._rope_args(q, k, v, rope_table, out, N)
+        _check(self._lib.blocklin_prefill_rope(self._handle, n_blocks, N // n_blocks, _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                                               _ptr(rope_table), _stream(k)), "blocklin_prefill_rope")
+        return o
+
+    def status(self) -> int:
+        """Synchronises the current stream; 0, or -6 if a bounded device-side wait of one of this cache's
+        launches ran out (``reset`` clears it)."""
+        st = ctypes.c_int(0)
+        _check(self._lib.blocklin_cache_status(self._handle, _stream(self.state), ctypes.byref(st)),
+               "blocklin_cache_status")
+        return st.value
 
     def peek(self, q, k, v, out=None):
         """Output of the block against cache + state(block) without committing (Algorithm 1's denoising steps)."""

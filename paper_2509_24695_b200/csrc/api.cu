@@ -99,14 +99,19 @@ size_t rope_workspace_need(const Problem& p) { return round256(rope_state_offset
 
 // Eq. 2 with its rotary factors: state from the rotated keys (z from the plain ones), apply with the rotated
 // queries (denominator from the plain ones).
+// `base` as in run_passes: the state that is added to (null: `state` itself); q may be null (state only).
 int run_rope(const Problem& p, const void* q, const void* k, const void* v, void* o, float* state, bool accumulate,
-             float eps, const __half2* rope, void* workspace, cudaStream_t stream) {
+             float eps, const __half2* rope, void* workspace, cudaStream_t stream, const float* base = nullptr) {
   if (umma_rope_supported(p)) {  // one launch on the tensor cores
-    UmmaCall c{k, v, q, o, state, nullptr, accumulate, eps, rope};
+    UmmaCall c{k, v, q, o, state, base, accumulate, eps, rope};
     return umma_run(p, c, workspace, stream);
   }
+  if (accumulate && base && base != state) {
+    if (cudaMemcpyAsync(state, base, state_bytes_of(p), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+      return LINATTN_ERR_CUDA;
+  }
   int st = cuda_status(fma_state(p, k, v, state, accumulate, partials_of(workspace), stream, rope));
-  if (st != LINATTN_OK) return st;
+  if (st != LINATTN_OK || !q) return st;
   return cuda_status(fma_apply(p, q, state, o, eps, stream, rope));
 }
 
@@ -180,6 +185,32 @@ static int step_impl(blocklin_cache* cache, const Problem& p, const void* q_blk,
   if (cache->workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
   if (p.N == 0) return LINATTN_OK;
   st = run_passes(p, k_blk, v_blk, q_blk, o_blk, cache->state, true, cache->eps, cache->workspace, stream);
+  if (st != LINATTN_OK) return st;
+  cache->blocks_seen += 1;
+  cache->tokens_seen += p.N;
+  return LINATTN_OK;
+}
+
+// One block with the rotary factors of Eq. 2.  commit: the cache takes the block (blocklin_step_rope); otherwise the
+// sum of cache and block goes to the state slot of the workspace and the cache is only read (blocklin_peek_rope).
+static int step_rope_impl(blocklin_cache* cache, const Problem& p, const void* q_blk, const void* k_blk,
+                          const void* v_blk, void* o_blk, const void* rope_table_blk, bool commit, cudaStream_t stream) {
+  if (p.d & 1) return LINATTN_ERR_UNSUPPORTED;
+  if ((q_blk == nullptr) != (o_blk == nullptr)) return LINATTN_ERR_INVALID_ARG;
+  if (p.N > 0 && (!k_blk || !v_blk || !rope_table_blk)) return LINATTN_ERR_INVALID_ARG;
+  if (o_blk && (o_blk == q_blk || o_blk == k_blk || o_blk == v_blk)) return LINATTN_ERR_INVALID_ARG;
+  int st = check_alignment(p, q_blk, k_blk, v_blk, o_blk);
+  if (st != LINATTN_OK) return st;
+  // the tensor-core kernel fetches the rotations in 16-byte chunks; the FMA kernels pair by pair
+  if (reinterpret_cast<uintptr_t>(rope_table_blk) & (umma_rope_supported(p) ? 15u : 3u)) return LINATTN_ERR_BAD_ALIGNMENT;
+  if (cache->workspace_bytes < rope_workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  if (p.N == 0) return LINATTN_OK;
+  const __half2* rope = static_cast<const __half2*>(rope_table_blk);
+  if (!commit) {
+    float* tmp = reinterpret_cast<float*>(static_cast<char*>(cache->workspace) + rope_state_offset(p));
+    return run_rope(p, q_blk, k_blk, v_blk, o_blk, tmp, true, cache->eps, rope, cache->workspace, stream, cache->state);
+  }
+  st = run_rope(p, q_blk, k_blk, v_blk, o_blk, cache->state, true, cache->eps, rope, cache->workspace, stream);
   if (st != LINATTN_OK) return st;
   cache->blocks_seen += 1;
   cache->tokens_seen += p.N;
@@ -266,6 +297,13 @@ int linattn_state_static_scratch(const linattn_desc* desc, int64_t N, const void
   if (cudaMemsetAsync(scratch, 0, LINATTN_WORKSPACE_CTRL_BYTES, (cudaStream_t)stream) != cudaSuccess)
     return LINATTN_ERR_CUDA;
   return run_passes(p, k, v, nullptr, nullptr, state, false, 0.f, scratch, (cudaStream_t)stream);
+}
+
+int linattn_static_scratch_status(void* stream, int* status) {
+  if (!status) return LINATTN_ERR_INVALID_ARG;
+  void* scratch = static_scratch_address();
+  if (!scratch) return LINATTN_ERR_CUDA;
+  return linattn_workspace_status(scratch, stream, status);
 }
 
 int linattn_apply(const linattn_desc* desc, int64_t N, const void* q, const float* state, void* o, float eps,
@@ -463,7 +501,15 @@ int blocklin_cache_reset(blocklin_cache* cache, void* stream) {
   if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
   cache->blocks_seen = 0;
   cache->tokens_seen = 0;
-  return cuda_status(cudaMemsetAsync(cache->state, 0, cache->state_bytes, (cudaStream_t)stream));
+  // the control block too: a recorded timeout and the barrier word it left half-counted go away with the past
+  cudaError_t e = cudaMemsetAsync(cache->state, 0, cache->state_bytes, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(cache->workspace, 0, LINATTN_WORKSPACE_CTRL_BYTES, (cudaStream_t)stream);
+  return cuda_status(e);
+}
+
+int blocklin_cache_status(const blocklin_cache* cache, void* stream, int* status) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  return linattn_workspace_status(cache->workspace, stream, status);
 }
 
 int blocklin_step(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
@@ -481,19 +527,40 @@ int blocklin_step_rope(blocklin_cache* cache, int64_t T_b, const void* q_blk, co
   Problem p;
   int st = resolve(&cache->desc, T_b, &p);
   if (st != LINATTN_OK) return st;
-  if (p.d & 1) return LINATTN_ERR_UNSUPPORTED;
-  if (p.N > 0 && (!q_blk || !k_blk || !v_blk || !o_blk || !rope_table_blk)) return LINATTN_ERR_INVALID_ARG;
-  if (o_blk && (o_blk == q_blk || o_blk == k_blk || o_blk == v_blk)) return LINATTN_ERR_INVALID_ARG;
-  if ((st = check_alignment(p, q_blk, k_blk, v_blk, o_blk)) != LINATTN_OK) return st;
-  if (!aligned16(rope_table_blk)) return LINATTN_ERR_BAD_ALIGNMENT;
-  if (cache->workspace_bytes < rope_workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
-  if (p.N == 0) return LINATTN_OK;
-  st = run_rope(p, q_blk, k_blk, v_blk, o_blk, cache->state, true, cache->eps, static_cast<const __half2*>(rope_table_blk),
-                cache->workspace, (cudaStream_t)stream);
+  return step_rope_impl(cache, p, q_blk, k_blk, v_blk, o_blk, rope_table_blk, true, (cudaStream_t)stream);
+}
+
+int blocklin_peek_rope(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
+                       void* o_blk, const void* rope_table_blk, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  Problem p;
+  int st = resolve(&cache->desc, T_b, &p);
   if (st != LINATTN_OK) return st;
-  cache->blocks_seen += 1;
-  cache->tokens_seen += p.N;
-  return LINATTN_OK;
+  if (p.N > 0 && (!q_blk || !o_blk)) return LINATTN_ERR_INVALID_ARG;
+  return step_rope_impl(cache, p, q_blk, k_blk, v_blk, o_blk, rope_table_blk, false, (cudaStream_t)stream);
+}
+
+int blocklin_prefill_rope(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,
+                          const void* v, void* o, const void* rope_table, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  if (n_blocks < 0 || T_b < 0) return LINATTN_ERR_INVALID_ARG;
+  if ((q == nullptr) != (o == nullptr)) return LINATTN_ERR_INVALID_ARG;
+  if (n_blocks == 0 || T_b == 0) return LINATTN_OK;
+  if (!k || !v || !rope_table) return LINATTN_ERR_INVALID_ARG;
+  Problem p;
+  int st = resolve(&cache->desc, n_blocks * T_b, &p);   // every block keeps the whole sequence's strides
+  if (st != LINATTN_OK) return st;
+  if ((st = check_alignment(p, q, k, v, o)) != LINATTN_OK) return st;
+  p.N = T_b;
+  const size_t esz = cache->desc.dtype == LINATTN_BF16 ? 2 : 4;
+  const size_t row = (size_t)(p.d / 2) * sizeof(__half2);   // one token's rotations
+  for (int64_t i = 0; i < n_blocks && st == LINATTN_OK; ++i) {
+    const size_t off = (size_t)(i * T_b) * (size_t)p.sn * esz;
+    st = step_rope_impl(cache, p, q ? static_cast<const char*>(q) + off : nullptr, static_cast<const char*>(k) + off,
+                        static_cast<const char*>(v) + off, o ? static_cast<char*>(o) + off : nullptr,
+                        static_cast<const char*>(rope_table) + (size_t)(i * T_b) * row, true, (cudaStream_t)stream);
+  }
+  return st;
 }
 
 int blocklin_peek(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
@@ -511,6 +578,35 @@ int blocklin_peek(blocklin_cache* cache, int64_t T_b, const void* q_blk, const v
   float* tmp = reinterpret_cast<float*>(static_cast<char*>(cache->workspace) + state_slot_offset(p));
   return run_passes(p, k_blk, v_blk, q_blk, o_blk, tmp, true, cache->eps, cache->workspace, (cudaStream_t)stream,
                     cache->state);
+}
+
+int blocklin_shard_state(blocklin_cache* cache, int64_t T_shard, const void* k_shard, const void* v_shard,
+                         float* state_out, int include_cache, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  Problem p;
+  int st = resolve(&cache->desc, T_shard, &p);
+  if (st != LINATTN_OK) return st;
+  if (!state_out || state_out == cache->state) return LINATTN_ERR_INVALID_ARG;
+  if (p.N > 0 && (!k_shard || !v_shard)) return LINATTN_ERR_INVALID_ARG;
+  if ((st = check_alignment(p, k_shard, v_shard, state_out, nullptr)) != LINATTN_OK) return st;
+  if (cache->workspace_bytes < workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (p.N == 0)   // a rank without tokens of this block contributes the cache (or nothing) alone
+    return cuda_status(include_cache ? cudaMemcpyAsync(state_out, cache->state, cache->state_bytes, cudaMemcpyDeviceToDevice, s)
+                                     : cudaMemsetAsync(state_out, 0, cache->state_bytes, s));
+  return run_passes(p, k_shard, v_shard, nullptr, nullptr, state_out, include_cache != 0, 0.f, cache->workspace, s,
+                    include_cache ? cache->state : nullptr);
+}
+
+int blocklin_shard_commit(blocklin_cache* cache, const float* state_in, int64_t block_tokens, void* stream) {
+  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
+  if (!state_in || block_tokens < 0) return LINATTN_ERR_INVALID_ARG;
+  if (state_in != cache->state &&
+      cudaMemcpyAsync(cache->state, state_in, cache->state_bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream) != cudaSuccess)
+    return LINATTN_ERR_CUDA;
+  cache->blocks_seen += 1;
+  cache->tokens_seen += block_tokens;
+  return LINATTN_OK;
 }
 
 int blocklin_prefill(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,

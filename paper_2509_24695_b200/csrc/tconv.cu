@@ -249,11 +249,14 @@ cudaError_t launch_step(const TconvParams& p, int B, cudaStream_t stream) {
   const long long tpb = (cols + 255) / 256, total = tpb * B;
   if (total >= (1ll << 31)) return cudaErrorInvalidValue;
   constexpr size_t smem = (size_t)kStepStages * kStepSegs * 256 * 16;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the opt-in to more than 48 KB of dynamic shared memory is a per-device setting of the kernel
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!attr_set[dev]) {
     const cudaError_t e = cudaFuncSetAttribute(tconv_step_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   const int sms = sm_count_of_device();
   if (!sms) return cudaErrorUnknown;
@@ -308,7 +311,9 @@ int run(const tconv_desc* d, long long T, long long T_b, const void* x, const fl
   dim3 grid((unsigned)((cols + 255) / 256), (unsigned)d->B);
   const bool few = T <= 3;
   cudaError_t e;
-  if (few && cache_in && y) {   // a block step of the paper's size: the staged kernel
+  // The staged kernel treats all T frames as ONE block (only the last frame gets the zero frame behind it), so it
+  // takes single blocks only; a prefill of several short blocks goes to the kernel that honours T_b.
+  if (few && T_b >= T && cache_in && y) {   // a block step of the paper's size: the staged kernel
     e = d->dtype == LINATTN_BF16 ? launch_step<__nv_bfloat16>(p, d->B, (cudaStream_t)stream)
                                  : launch_step<float>(p, d->B, (cudaStream_t)stream);
   } else {

@@ -1400,12 +1400,15 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
     mq = mk; mo = mk;  // never dereferenced
   }
   if (!do_state) { mk = mq; mv = mq; }
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the opt-in to more than 48 KB of dynamic shared memory is a per-device setting of the kernel
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LINATTN_ERR_CUDA;
+  if (!attr_set[dev]) {
     if (cudaFuncSetAttribute(umma_fused_kernel<D, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM) !=
         cudaSuccess)
       return LINATTN_ERR_CUDA;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   void* args[] = {&mk, &mv, &mq, &mo, &fp};
   const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D, ROPE>, dim3(grid), dim3(Roles<ROPE>::THREADS), args,

@@ -74,7 +74,15 @@ def test_sizes_and_validation_without_gpu(lib):
 
 
 def test_product_package_does_not_touch_the_oracle():
-    """The oracle is test infrastructure: nothing under the package may import or load it."""
+    """The oracle and the seeded input generator are test infrastructure: nothing under the package may import
+    or load them (and neither of the two imports the other or the package)."""
+    for mod, banned in (("oracle", ("import synth", "paper_2509_24695_b200", "libsynth")),
+                        ("synth", ("import oracle", "from oracle", "paper_2509_24695_b200", "liblinattn"))):
+        for dirpath, _, files in os.walk(os.path.join(ROOT, mod)):
+            for f in files:
+                if f.endswith((".py", ".c", ".h")):
+                    text = open(os.path.join(dirpath, f)).read()
+                    assert not any(b in text for b in banned), (mod, f)
     pkg = os.path.join(ROOT, "paper_2509_24695_b200")
     for dirpath, _, files in os.walk(pkg):
         if "_build" in dirpath:
@@ -83,6 +91,7 @@ def test_product_package_does_not_touch_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".c", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in text and "from oracle" not in text and "liblinattn_oracle" not in text, f
+                assert "import synth" not in text and "libsynth" not in text, f
 
 
 def test_tconv_sizes_and_validation_without_gpu(lib):

@@ -8,7 +8,7 @@ tile edges, seeded random picks) against the oracle's apply of ITS OWN state to 
 import numpy as np
 import pytest
 
-from paper_2509_24695_b200 import synth
+import synth
 from parity_util import assert_parity_bf16, assert_state_close, sample_rows, to_dev, to_f64
 
 pytestmark = pytest.mark.gpu

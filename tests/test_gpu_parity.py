@@ -4,7 +4,7 @@ for the oracle to finish in seconds; the full-size workloads are in test_gpu_ful
 import numpy as np
 import pytest
 
-from paper_2509_24695_b200 import synth
+import synth
 from parity_util import assert_parity_bf16, assert_parity_f32, assert_state_close, to_dev, to_f64
 
 pytestmark = pytest.mark.gpu

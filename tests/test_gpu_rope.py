@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from paper_2509_24695_b200 import synth
+import synth
 from parity_util import assert_parity_bf16, assert_parity_f32, to_dev, to_f64
 
 pytestmark = pytest.mark.gpu
@@ -104,3 +104,89 @@ def test_rope_block_steps_match_the_block_causal_oracle(la, orc, case):
     full = la.linattn_forward_rope(to_dev(q), to_dev(k), to_dev(v), table, EPS)
     last = (N - 1) // T_b * T_b
     check(to_f64(stepped[:, last:]), to_f64(full[:, last:]).copy(), "last block vs bidirectional rotary forward")
+
+
+def tdtype(dtype):
+    import torch
+
+    return torch.bfloat16 if dtype == "bf16" else torch.float32
+
+
+def packed_table(la, T, Hh, Ww, d):
+    cos, sin = synth.rope_table(T, Hh, Ww, d)
+    table = la.rope_pack(to_dev(cos), to_dev(sin))
+    packed = table.cpu().numpy().astype(np.float64)
+    return table, packed[..., 0], packed[..., 1]
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 112), ("f32", 112), ("bf16", 64), ("bf16", 6)])
+def test_rope_denoise_loop_reads_without_committing(la, orc, dtype, d):
+    """Algorithm 1 on the attention the model runs (Eq. 2 with RoPE): every denoising step of a block reads the
+    rotary cache together with the noisy block itself and leaves the cache as it was; only the clean block is
+    committed.  The oracle's step runs on a copy of its cache."""
+    import torch
+
+    B, H, (T, Hh, Ww), fb, M, steps = 1, 3, (6, 10, 15), 2, 3, 2    # blocks of fb = 2 frames = 300 tokens
+    T_b = fb * Hh * Ww
+    table, cs, sn = packed_table(la, T, Hh, Ww, d)
+    check = assert_parity_bf16 if dtype == "bf16" else assert_parity_f32
+    cache = la.BlockLinCache(B, H, d, tdtype(dtype), "cuda", max_T_b=T_b, eps=EPS)
+    ocache = orc.new_cache(B, H, d)
+    for blk in range(M):
+        sl = slice(blk * T_b, (blk + 1) * T_b)
+        tab = table[sl].contiguous()
+        before = cache.state.clone()
+        for j in range(steps):          # noisy versions of the block: other values each time, same positions
+            q, k, v = gen(B, T_b, H, d, 5400 + 10 * blk + j, dtype)
+            o = cache.peek_rope(to_dev(q), to_dev(k), to_dev(v), tab)
+            ref = orc.rope_block_step((ocache[0].copy(), ocache[1].copy()), q, k, v, cs[sl], sn[sl], EPS)
+            check(to_f64(o), ref, f"rotary peek block {blk} step {j}")
+            assert torch.equal(cache.state, before), "a read-only step changed the cache"
+            assert cache.info()["blocks_seen"] == blk
+        q, k, v = gen(B, T_b, H, d, 5500 + blk, dtype)               # the clean block
+        o_peek = cache.peek_rope(to_dev(q), to_dev(k), to_dev(v), tab)
+        o_step = cache.step_rope(to_dev(q), to_dev(k), to_dev(v), tab)
+        assert torch.equal(o_peek, o_step)                            # same arithmetic, committed or not
+        check(to_f64(o_step), orc.rope_block_step(ocache, q, k, v, cs[sl], sn[sl], EPS), f"rotary step block {blk}")
+        S, z = ocache
+        got = to_f64(cache.state)
+        # z sums the plain features in fp32.  S sums rotated features: fp32 throughout on the fp32 path; on the bf16
+        # path the rotated key is rounded to bf16 before it enters the tensor core (2^-9 relative per term, unbiased:
+        # the sum's error is about 1.5e-3 of the state's RMS, its largest of 37 632 entries several times that)
+        for g, r, name, rel in ((got[..., :d, :].swapaxes(-1, -2), S, "S", 1e-5 if dtype == "f32" else 1e-2),
+                                (got[..., d, :], z, "z", 1e-5)):
+            rms = np.sqrt((r ** 2).mean(axis=tuple(range(2, r.ndim)), keepdims=True))
+            assert (np.abs(g - r) <= rel * (np.abs(r) + rms)).all(), f"rotary cache after block {blk}: {name}"
+    assert cache.info()["blocks_seen"] == M and cache.status() == 0
+
+
+@pytest.mark.parametrize("case", [("bf16", 3, 112, (6, 6, 10), 2), ("f32", 2, 112, (4, 5, 5), 1), ("bf16", 2, 64, (6, 4, 8), 3),
+                                  ("bf16", 2, 6, (4, 3, 5), 2)],
+                         ids=lambda c: "%s_H%d_d%d_fb%d" % (c[0], c[1], c[2], c[4]))
+def test_rope_prefill_equals_steps_and_oracle(la, orc, case):
+    """blocklin_prefill_rope over all blocks: the bits of single rotary steps, the oracle's block-causal rotary form,
+    and (absorb only: q = o = NULL) the same cache."""
+    import torch
+
+    dtype, H, d, (T, Hh, Ww), fb = case
+    B, N, T_b = 2, T * Hh * Ww, fb * Hh * Ww
+    M = N // T_b
+    q, k, v = gen(B, N, H, d, 5600 + N + d, dtype)
+    table, cs, sn = packed_table(la, T, Hh, Ww, d)
+    qd, kd, vd = to_dev(q), to_dev(k), to_dev(v)
+    check = assert_parity_bf16 if dtype == "bf16" else assert_parity_f32
+    cache = la.BlockLinCache(B, H, d, tdtype(dtype), "cuda", max_T_b=T_b, eps=EPS, strides=tuple(qd.stride()[:3]))
+    stepped = torch.empty_like(qd)       # blocks are token ranges of the long tensors: they keep its batch stride
+    for i in range(M):
+        sl = slice(i * T_b, (i + 1) * T_b)
+        cache.step_rope(qd[:, sl], kd[:, sl], vd[:, sl], table[sl], out=stepped[:, sl])
+    final = cache.state.clone()
+    cache.reset()
+    assert (cache.state == 0).all()
+    o = cache.prefill_rope(qd, kd, vd, table, M)
+    assert torch.equal(o, stepped) and torch.equal(cache.state, final)
+    assert cache.info() == {"blocks_seen": M, "tokens_seen": N, "state_bytes": B * H * (d * d + d) * 4}
+    check(to_f64(o), orc.rope_forward(q, k, v, cs, sn, EPS, T_b=T_b), f"rotary prefill {case}")
+    cache.reset()
+    assert cache.prefill_rope(None, kd, vd, table, M) is None        # context only
+    assert torch.equal(cache.state, final) and cache.status() == 0

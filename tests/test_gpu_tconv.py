@@ -10,7 +10,7 @@ import numpy as np
 import pytest
 
 from oracle import tconv as orc_conv
-from paper_2509_24695_b200 import synth
+import synth
 from parity_util import to_dev, to_f64
 
 pytestmark = pytest.mark.gpu
@@ -64,6 +64,9 @@ CASES = [
     (1, 4, 9, 2240, 1),     # the model width
     (3, 3, 5, 8, 3),
     (1, 1, 11, 24, 1),      # a single frame
+    (1, 3, 9, 16, 1),       # three one-frame blocks in one prefill: every block ends with the zero frame
+    (2, 2, 9, 16, 1),       # two one-frame blocks, two batch entries
+    (1, 3, 130, 40, 3),     # one three-frame block: the short-step kernel
 ]
 
 

@@ -14,7 +14,7 @@ import numpy as np
 import pytest
 
 import oracle as oracle_mod
-from paper_2509_24695_b200 import synth
+import synth
 
 EPS = 1e-6
 
@@ -317,6 +317,70 @@ def pin_rope_closed_form_d2(o):
     assert np.allclose(out[0, 0, 0], [0.0, -1.0], atol=1e-14)
 
 
+def pin_rope_block_causal_closed_form_d2(o):
+    """d = 2, phi(q) = phi(k) = (1, 0), blocks of T_b tokens: token n sees the tokens of its own and of earlier
+    blocks, the rotated dot product is cos(theta_n - theta_m) and the plain one is 1, so
+    o_n = sum_{m visible} cos(theta_n - theta_m) v_m / (count_n + eps)  (Eq. 3's running sums on Eq. 2's
+    right-hand form).  Fixes the block-causal rotary form against the mathematics in all three ways the oracle
+    computes it: block by block, masked brute force, and cached steps on a caller-held cache."""
+    N, T_b, eps = 11, 4, 0.5                      # blocks of 4, 4 and 3 tokens
+    th = np.array([0.0, 0.3, -1.1, 2.0, np.pi / 2, -0.4, 1.7, 0.9, -2.5, 0.05, 3.0])
+    q = np.zeros((1, N, 1, 2)); q[..., 0] = 1.0; q[..., 1] = -3.0     # the negative entry is cut by the ReLU
+    k = q.copy()
+    v = _rand((1, N, 1, 2), 91, 3)
+    blk = np.arange(N) // T_b
+    visible = blk[None, :] <= blk[:, None]                            # [n, m]
+    want = ((np.cos(th[:, None] - th[None, :]) * visible) @ v[0, :, 0]) / (visible.sum(1) + eps)[:, None]
+    cs, sn = np.cos(th)[:, None], np.sin(th)[:, None]
+    assert np.allclose(o.rope_forward(q, k, v, cs, sn, eps, T_b=T_b)[0, :, 0], want, rtol=0, atol=1e-14)
+    assert np.allclose(o.rope_forward(q, k, v, cs, sn, eps, quadratic=True, T_b=T_b)[0, :, 0], want, rtol=0, atol=1e-14)
+    cache = o.new_cache(1, 1, 2)
+    for n0 in range(0, N, T_b):
+        sl = slice(n0, min(n0 + T_b, N))
+        args = (q[:, sl].copy(), k[:, sl].copy(), v[:, sl].copy(), cs[sl], sn[sl], eps)
+        # a denoising step of Algorithm 1 reads the cache without committing: the step on a copy
+        peek = o.rope_block_step((cache[0].copy(), cache[1].copy()), *args)
+        before = (cache[0].copy(), cache[1].copy())
+        out = o.rope_block_step(cache, *args)
+        assert np.array_equal(peek, out)
+        assert np.allclose(out[0, :, 0], want[sl], rtol=0, atol=1e-14)
+        assert not np.array_equal(before[1], cache[1])                # the committing step did change the cache
+    # the cache after the last block, in closed form: z = (N, 0); S = sum_m (cos, sin)(theta_m)^T v_m
+    S, z = cache
+    assert np.array_equal(z[0, 0], [N, 0.0])
+    assert np.allclose(S[0, 0], np.stack([np.cos(th), np.sin(th)], 0) @ v[0, :, 0], rtol=0, atol=1e-14)
+    # commit only (no output) leaves the same cache
+    c2 = o.new_cache(1, 1, 2)
+    for n0 in range(0, N, T_b):
+        sl = slice(n0, min(n0 + T_b, N))
+        assert o.rope_block_step(c2, q[:, sl].copy(), k[:, sl].copy(), v[:, sl].copy(), cs[sl], sn[sl], eps, want_o=False) is None
+    assert np.array_equal(c2[0], S) and np.array_equal(c2[1], z)
+
+
+def pin_rope_steps_equal_one_shot(o):
+    """Cached rotary steps over several heads and batch entries equal the one-shot block-causal form, and a
+    step's table rows are the block's own: shifting them by one token changes the result."""
+    B, N, H, d, T_b = 2, 10, 3, 6, 4
+    q, k, v = _qkv(B, N, H, d, 95)
+    cs, sn, _ = _angles(N, d // 2, 96)
+    ref = o.rope_forward(q, k, v, cs, sn, EPS, T_b=T_b)
+    cache = o.new_cache(B, H, d)
+    for n0 in range(0, N, T_b):
+        sl = slice(n0, min(n0 + T_b, N))
+        out = o.rope_block_step(cache, q[:, sl].copy(), k[:, sl].copy(), v[:, sl].copy(), cs[sl], sn[sl], EPS)
+        assert np.allclose(out, ref[:, sl], rtol=1e-12, atol=1e-13)
+    sl = slice(4, 8)
+    c0 = o.new_cache(B, H, d)
+    a = o.rope_block_step(c0, q[:, sl].copy(), k[:, sl].copy(), v[:, sl].copy(), cs[sl], sn[sl], EPS)
+    c1 = o.new_cache(B, H, d)
+    b = o.rope_block_step(c1, q[:, sl].copy(), k[:, sl].copy(), v[:, sl].copy(), cs[5:9], sn[5:9], EPS)
+    assert np.abs(a - b).max() > 1e-3
+    # units are independent and land in their own slice of the cache
+    c3 = o.new_cache(1, 1, d)
+    o.rope_block_step(c3, q[1:, sl, 2:].copy(), k[1:, sl, 2:].copy(), v[1:, sl, 2:].copy(), cs[sl], sn[sl], EPS)
+    assert np.array_equal(c3[0][0, 0], c0[0][1, 2]) and np.array_equal(c3[1][0, 0], c0[1][1, 2])
+
+
 def pin_rope_reduces_to_plain(o):
     """Zero angles, or one common angle per feature pair for all tokens (relative angle zero), give Eq. 2
     without rotary factors: the numerator only sees angle differences and the denominator sees none."""
@@ -370,7 +434,8 @@ def pin_rope_linear_equals_quadratic_and_shift(o):
 PINS = [pin_hand_worked_example, pin_golden_hand_worked_d2, pin_exact_rational, pin_linear_equals_quadratic, pin_bf16_decode_and_tiny_config,
         pin_constant_v, pin_single_token, pin_one_hot_is_segment_mean, pin_invariances, pin_sign, pin_convexity,
         pin_block_forms_agree, pin_cache_size_constant, pin_strides_and_rows, pin_rope_closed_form_d2,
-        pin_rope_reduces_to_plain, pin_rope_linear_equals_quadratic_and_shift]
+        pin_rope_reduces_to_plain, pin_rope_linear_equals_quadratic_and_shift, pin_rope_block_causal_closed_form_d2,
+        pin_rope_steps_equal_one_shot]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -421,8 +486,16 @@ MUTANTS = {
     "rope_quadratic_den_rotated": ("wden += qp[i] * kp[i];", "wden += qr[i] * kr[i];"),
     "rope_block_mask_off": ("if (T_b > 0 && (m / T_b) > (n / T_b)) continue; /* later block: not visible (T_b <= 0: no mask) */",
                             "if (T_b > 0 && (m / T_b) >= (n / T_b)) continue;"),
-    "rope_block_reads_before_commit": ("      for (int64_t n = n0; n < n1; ++n) { /* commit the block ... */",
-                                       "      for (int64_t n = n0; n < n0; ++n) { /* commit the block ... */"),
+    "rope_block_reads_before_commit": ("  for (int64_t n = n0; n < n1; ++n) { /* commit the block ... */",
+                                       "  for (int64_t n = n0; n < n0; ++n) { /* commit the block ... */"),
+    "rope_block_forgets_past": ("      rope_block(s, q, k, v, cs, sn, b, h, n0, n1, eps, S, z, z + d, z + 2 * d, o);",
+                                "      memset(S, 0, sizeof(double) * (d * d + d));\n"
+                                "      rope_block(s, q, k, v, cs, sn, b, h, n0, n1, eps, S, z, z + d, z + 2 * d, o);"),
+    "rope_step_unit_offset": ("S + u * d * d, z + u * d, tmp, tmp + d, o);", "S + u * d, z + u * d, tmp, tmp + d, o);"),
+    "rope_step_cache_zeroed": ("    double* tmp = (double*)calloc((size_t)(2 * d), sizeof(double));\n    rope_block(",
+                               "    double* tmp = (double*)calloc((size_t)(2 * d), sizeof(double));\n"
+                               "    memset(z + u * d, 0, sizeof(double) * d);\n    rope_block("),
+    "rope_step_first_head_only": ("u / s->H, u % s->H, 0, s->N, eps,", "u / s->H, 0, 0, s->N, eps,"),
     "rope_token_index": ("rope_features(s, k, base, cs, sn, n, plain, rot);", "rope_features(s, k, base, cs, sn, 0, plain, rot);"),
 }
 

@@ -12,7 +12,7 @@ import ctypes
 import numpy as np
 import pytest
 
-from paper_2509_24695_b200 import synth
+import synth
 from parity_util import assert_state_close, to_dev, to_f64
 
 pytestmark = pytest.mark.gpu
@@ -29,12 +29,12 @@ def la():
     return la
 
 
-def _state_both_ways(la, shape, seed, dtype="bf16"):
+def _state_both_ways(la, shape, seed, dtype="bf16", kv=None):
     import torch
 
     B, N, H, d = shape
-    k = to_dev(synth.gauss(shape, seed, 2, dtype=dtype))
-    v = to_dev(synth.gauss(shape, seed, 3, dtype=dtype))
+    k = to_dev(synth.gauss(shape, seed, 2, dtype=dtype) if kv is None else kv[0])
+    v = to_dev(synth.gauss(shape, seed, 3, dtype=dtype) if kv is None else kv[1])
     ref = la.linattn_state(k, v)
     out = torch.full((B, H, d + 1, d), float("nan"), dtype=torch.float32, device="cuda")
     lib = la.load_library()
@@ -44,6 +44,9 @@ def _state_both_ways(la, shape, seed, dtype="bf16"):
                                               ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
     assert status == 0, lib.linattn_status_string(status)
     torch.cuda.synchronize()
+    assert la.static_scratch_status() == 0          # no bounded wait ran out in the launch just made
+    # same kernel, same work split, same order of the partial sums: the two entry points agree bit for bit
+    assert torch.equal(out, ref), "the built-in scratch changed the result"
     return to_f64(out), to_f64(ref)
 
 
@@ -55,6 +58,17 @@ def test_two_calls_in_a_row_match_linattn_state(la):
         d = shape[3]
         assert np.isfinite(got).all()
         assert_state_close(got, ref[..., :d, :].swapaxes(-1, -2), ref[..., d, :], 1e-5, f"static scratch {shape}")
+
+
+def test_small_integers_match_the_oracle_bit_for_bit(la, orc):
+    # inputs in {-2..2}: every partial sum is an integer below 2^24, so the fp32 state must equal the fp64
+    # oracle's exactly, whatever the order of the sums -- twice in a row through the shared array
+    for shape, seed in (((1, 3000, 5, 112), 4111), ((2, 1200, 3, 64), 4112)):
+        k, v = synth.smallint(shape, seed, 2, 2), synth.smallint(shape, seed, 3, 2)
+        got, _ = _state_both_ways(la, shape, seed, kv=(k, v))
+        S, z = orc.state(k, v)
+        d = shape[3]
+        assert np.array_equal(got[..., :d, :].swapaxes(-1, -2), S) and np.array_equal(got[..., d, :], z), shape
 
 
 def test_other_paths_and_repeat(la):
@@ -76,6 +90,13 @@ def test_too_large_is_refused_and_zero_tokens_is_an_empty_sum(la):
     with pytest.raises(la.LinAttnError) as e:
         la.linattn_state_static_scratch(k, k.clone(), out)
     assert e.value.status == -8
+    # fp32 inputs keep one partial state per 512 tokens: 20 heads of dimension 112 fit up to 8192 tokens
+    kf = torch.zeros((1, 8193, 20, 112), dtype=torch.float32, device="cuda")
+    outf = torch.zeros((1, 20, 113, 112), dtype=torch.float32, device="cuda")
+    with pytest.raises(la.LinAttnError) as e:
+        la.linattn_state_static_scratch(kf, kf.clone(), outf)
+    assert e.value.status == -8
+    la.linattn_state_static_scratch(kf[:, :8192], kf[:, :8192].clone(), outf)
     k0 = torch.zeros((1, 0, 2, 112), dtype=torch.bfloat16, device="cuda")
     out0 = torch.ones((1, 2, 113, 112), dtype=torch.float32, device="cuda")
     la.linattn_state_static_scratch(k0, k0.clone(), out0)
