@@ -359,32 +359,55 @@ class BlockLinCache:
     """
 
     def __init__(self, B: int, H: int, d: int, dtype, device, max_T_b: int, eps: float = 1e-6,
-                 strides: tuple[int, int, int] = (0, 0, 0), prefill_blocks: int = 0):
+                 strides: tuple[int, int, int] = (0, 0, 0), prefill_blocks: int = 0, state=None, workspace=None):
+        """state / workspace: caller-provided device tensors (a float32 ``[B, H, d+1, d]`` tensor and a uint8 tensor
+        of at least ``workspace_bytes_needed`` bytes, both 16-byte aligned) for callers that manage their own
+        pools; by default both are allocated here with torch."""
         torch = _torch()
         self._lib = load_library()
         code = LINATTN_BF16 if dtype == torch.bfloat16 else LINATTN_F32 if dtype == torch.float32 else None
         if code is None:
             raise TypeError(f"unsupported dtype {dtype}")
         self._desc = _Desc(B, H, d, code, *strides)
-        sb, wb = ctypes.c_size_t(), ctypes.c_size_t()
-        _check(self._lib.blocklin_cache_bytes(ctypes.byref(self._desc), max_T_b, ctypes.byref(sb), ctypes.byref(wb)),
-               "blocklin_cache_bytes")
-        self.state = torch.empty((B, H, d + 1, d), dtype=torch.float32, device=device)
-        assert self.state.numel() * 4 == sb.value
-        nbytes = wb.value
-        if prefill_blocks > 1:  # room for prefill() to process that many blocks of max_T_b tokens together
-            pb = ctypes.c_size_t()
-            _check(self._lib.blocklin_prefill_workspace_bytes(ctypes.byref(self._desc), prefill_blocks, max_T_b,
-                                                              ctypes.byref(pb)), "blocklin_prefill_workspace_bytes")
-            nbytes = max(nbytes, pb.value)
-        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        state_bytes_, nbytes = self.sizes(B, H, d, dtype, max_T_b, prefill_blocks, strides)
+        if state is None:
+            state = torch.empty((B, H, d + 1, d), dtype=torch.float32, device=device)
+        elif tuple(state.shape) != (B, H, d + 1, d) or state.dtype != torch.float32 or not state.is_contiguous():
+            raise ValueError("state must be a contiguous float32 [B, H, d+1, d] tensor")
+        self.state = state
+        assert self.state.numel() * 4 == state_bytes_
+        self.workspace_bytes_needed = nbytes
+        if workspace is None:
+            workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        elif workspace.dtype != torch.uint8 or workspace.numel() < nbytes or not workspace.is_contiguous():
+            raise ValueError(f"workspace must be a contiguous uint8 tensor of at least {nbytes} bytes")
+        else:
+            nbytes = workspace.numel()
+        self.workspace = workspace
         self.max_T_b, self.eps = max_T_b, eps
         self._handle = ctypes.c_void_p()
         _check(self._lib.blocklin_cache_init(ctypes.byref(self._handle), ctypes.byref(self._desc), eps,
-                                             _ptr(self.state), sb.value, _ptr(self.workspace), nbytes,
+                                             _ptr(self.state), state_bytes_, _ptr(self.workspace), nbytes,
                                              _stream(self.state)), "blocklin_cache_init")
         if prefill_blocks > 1:
             _check(self._lib.blocklin_cache_joint_prefill(self._handle, 1), "blocklin_cache_joint_prefill")
+
+    @staticmethod
+    def sizes(B: int, H: int, d: int, dtype, max_T_b: int, prefill_blocks: int = 0, strides=(0, 0, 0)) -> tuple[int, int]:
+        """(state bytes, workspace bytes) a cache of this shape needs; prefill_blocks > 1: room for ``prefill`` to
+        take that many blocks of max_T_b tokens together."""
+        torch = _torch()
+        lib = load_library()
+        desc = _Desc(B, H, d, LINATTN_BF16 if dtype == torch.bfloat16 else LINATTN_F32, *strides)
+        sb, wb = ctypes.c_size_t(), ctypes.c_size_t()
+        _check(lib.blocklin_cache_bytes(ctypes.byref(desc), max_T_b, ctypes.byref(sb), ctypes.byref(wb)), "blocklin_cache_bytes")
+        nbytes = wb.value
+        if prefill_blocks > 1:
+            pb = ctypes.c_size_t()
+            _check(lib.blocklin_prefill_workspace_bytes(ctypes.byref(desc), prefill_blocks, max_T_b, ctypes.byref(pb)),
+                   "blocklin_prefill_workspace_bytes")
+            nbytes = max(nbytes, pb.value)
+        return sb.value, nbytes
 
     def reset(self):
         _check(self._lib.blocklin_cache_reset(self._handle, _stream(self.state)), "blocklin_cache_reset")
@@ -547,10 +570,12 @@ def tconv_forward(x, w, out=None):
 class TConvCache:
     """The conv cache of the block-causal Mix-FFN: the last frame of the previous block, [B, HW, D]."""
 
-    def __init__(self, B: int, HW: int, D: int, dtype, device):
+    def __init__(self, B: int, HW: int, D: int, dtype, device, frame=None):
         torch = _torch()
         self._lib = load_library()
-        self.frame = torch.empty((B, HW, D), dtype=dtype, device=device)
+        if frame is not None and (tuple(frame.shape) != (B, HW, D) or frame.dtype != dtype or not frame.is_contiguous()):
+            raise ValueError("frame must be a contiguous [B, HW, D] tensor of the cache's dtype")
+        self.frame = torch.empty((B, HW, D), dtype=dtype, device=device) if frame is None else frame
         nbytes = ctypes.c_size_t()
         _check(self._lib.tconv_cache_bytes(ctypes.byref(self._desc(0)), ctypes.byref(nbytes)), "tconv_cache_bytes")
         assert nbytes.value == self.frame.numel() * self.frame.element_size()

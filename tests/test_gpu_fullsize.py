@@ -58,6 +58,31 @@ def test_720p_head_dim_sweep(la, orc, d):
     _check_bidirectional(la, orc, synth.p720_sweep(d), n_rows=48)
 
 
+@pytest.mark.parametrize("name", ["480p", "720p"])
+def test_fp32_io_path_at_layer_size(la, orc, name):
+    """The fp32 I/O path at the 480p / 720p token counts (where every split-N chunk accumulates ~500-1200 tokens in
+    fp32): whole state and sampled output rows within 1e-5 of the oracle.  Same seeded draws as the bf16 layers,
+    kept as float32 values."""
+    import torch
+
+    from parity_util import assert_parity_f32
+
+    w = synth.P480 if name == "480p" else synth.P720
+    shape = (w.B, w.N, w.H, w.d)
+    q, k, v = (synth.gauss(shape, w.seed, t, scale=w.scale, dtype="f32") for t in (1, 2, 3))
+    qd, kd, vd = to_dev(q), to_dev(k), to_dev(v)
+    ws = la.new_workspace(qd)
+    o = la.linattn_forward(qd, kd, vd, w.eps, workspace=ws)
+    st = la.linattn_state(kd, vd, workspace=ws)
+    assert la.workspace_status(ws) == 0
+    S, z = orc.state(k, v)
+    assert_state_close(to_f64(st), S, z, 1e-5, f"{w.name} fp32 state")
+    rows = sample_rows(w.N, 64, w.seed + 1)
+    ref = orc.apply_rows(q, S, z, w.eps, rows)
+    assert_parity_f32(to_f64(o[:, torch.from_numpy(rows).cuda()]), ref, f"{w.name} fp32 sampled rows")
+    assert torch.isfinite(o).all() and (o.abs().amax(dim=(0, 2, 3)) > 0).all()
+
+
 def test_480p_block_causal_seven_steps(la, orc):
     """Config 4 at full size: 7 steps of 4680 tokens against the oracle's block-wise prefix states."""
     import torch
