@@ -41,8 +41,12 @@
  * Pins (tests/test_oracle_pins.py): closed forms (constant V, N = 1, one-hot
  * features = segment mean), an exact rational worked example, brute-force
  * equality of the linear, quadratic, masked and stepped forms, invariances
- * (positive scaling, permutation, sign of negative entries), convexity, and
- * a mutation test showing that planted mistakes fail those pins.
+ * (positive scaling, permutation, sign of negative entries), convexity; for
+ * the rotary forms the closed form sum_m cos(theta_n - theta_m) v_m / (count
+ * + eps) at d = 2, over all tokens and over the tokens a block may see, for
+ * the one-shot, the masked brute-force and the cached-step functions alike;
+ * and a mutation test showing that planted mistakes fail those pins.  No
+ * function here is unpinned.
  *
  * Tensor layout: element (b, n, h, e) of Q/K/V/O lives at
  *   b*stride_b + n*stride_n + h*stride_h + e   (strides in elements).

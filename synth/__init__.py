@@ -163,25 +163,37 @@ def qkv_block(w: Workload, blk: int, dtype: str = "bf16", n_tokens: int | None =
     return tuple(outs)
 
 
-def rope_table(T: int, Hh: int, Ww: int, d: int, base: float = 10000.0):
-    """cos, sin tables ``[T*Hh*Ww, d//2]`` (float32) of a 3D rotary embedding for tokens ordered (t, h, w).
+def rope_axes(T: int, Hh: int, Ww: int, d: int, base: float = 10000.0, split=None):
+    """Per-axis cos, sin tables of a 3D rotary embedding: ``((cos_t, sin_t), (cos_h, sin_h), (cos_w, sin_w), (pt, ph, pw))``
+    with cos_a, sin_a of shape ``[positions of axis a, pairs of axis a]`` (float32).
 
     The paper gives neither the split of the head dim over the three axes nor the base frequency, so this
     is only a plausible input for tests and measurements: of the d//2 feature pairs, d//6 go to the height
-    and to the width axis each and the rest to time; pair i of an axis with n_a pairs turns by
-    ``pos * base**(-i / n_a)`` (the rotary formula of Su et al., per axis).
+    and to the width axis each and the rest to time (or ``split = (pt, ph, pw)``); pair i of an axis with n_a
+    pairs turns by ``pos * base**(-i / n_a)`` (the rotary formula of Su et al., per axis).
     """
     half = d // 2
-    n_hw = d // 6
-    n_t = half - 2 * n_hw
-    t, h, w = np.meshgrid(np.arange(T), np.arange(Hh), np.arange(Ww), indexing="ij")
-    cols = []
-    for pos, n_a in ((t, n_t), (h, n_hw), (w, n_hw)):
+    if split is None:
+        n_hw = d // 6
+        split = (half - 2 * n_hw, n_hw, n_hw)
+    assert sum(split) == half
+    out = []
+    for n_pos, n_a in zip((T, Hh, Ww), split):
         freq = base ** (-np.arange(n_a, dtype=np.float64) / max(n_a, 1))
-        cols.append(pos.reshape(-1, 1).astype(np.float64) * freq[None, :])
-    theta = np.concatenate(cols, axis=1)
-    assert theta.shape == (T * Hh * Ww, half)
-    return np.cos(theta).astype(np.float32), np.sin(theta).astype(np.float32)
+        theta = np.arange(n_pos, dtype=np.float64)[:, None] * freq[None, :]
+        out.append((np.cos(theta).astype(np.float32), np.sin(theta).astype(np.float32)))
+    return out[0], out[1], out[2], tuple(split)
+
+
+def rope_table(T: int, Hh: int, Ww: int, d: int, base: float = 10000.0, split=None):
+    """cos, sin tables ``[T*Hh*Ww, d//2]`` (float32) of the same embedding spelled out per token, tokens ordered
+    (t, h, w): pairs [0, pt) follow t, [pt, pt+ph) follow h, the rest follow w (see ``rope_axes``)."""
+    axes = rope_axes(T, Hh, Ww, d, base, split)
+    t, h, w = np.meshgrid(np.arange(T), np.arange(Hh), np.arange(Ww), indexing="ij")
+    cos = np.concatenate([axes[a][0][pos.reshape(-1)] for a, pos in enumerate((t, h, w))], axis=1)
+    sin = np.concatenate([axes[a][1][pos.reshape(-1)] for a, pos in enumerate((t, h, w))], axis=1)
+    assert cos.shape == (T * Hh * Ww, d // 2)
+    return np.ascontiguousarray(cos), np.ascontiguousarray(sin)
 
 
 # ---- inputs of the temporal convolution of the Mix-FFN: x[B, T, HW, D] frames and per-channel taps w[3, D] ----
