@@ -135,36 +135,6 @@ LINATTN_API int linattn_forward_rope(const linattn_desc* desc, int64_t N, const 
                                      void* o, float eps, const void* rope_table, void* workspace,
                                      size_t workspace_bytes, void* stream);
 
-/* Eq. 2 with rotary factors that follow a token's (frame, row, column) position one axis at a time: the 3D RoPE of
- * Sec. 3.1 ("Linear Attention in Video DiT").  The tokens are those of a T x Hh x Ww latent grid in frame-major
- * order (token n = (t*Hh + h)*Ww + w); feature pairs [0, pt) turn with t, [pt, pt+ph) with h, [pt+ph, d/2) with w
- * (pt + ph + pw = d/2; which split and which frequencies is the caller's choice, the paper does not print them).
- * Same operation as linattn_forward_rope with the per-token table that these per-axis rotations spell out, but
- * the rotations come as three small tables (T*pt + Hh*ph + Ww*pw entries) that stay on chip, where a per-token
- * table is as many bytes again as Q or K.  Tensor-core path only: bf16, d = 112 (the model's head dim); other
- * shapes return LINATTN_ERR_UNSUPPORTED and use the per-token table.  A split in which all three axes meet inside
- * one group of four pairs (4c .. 4c+3) is LINATTN_ERR_UNSUPPORTED as well.
- *
- * linattn_rope3d is HOST data; `table` is a DEVICE buffer of linattn_rope3d_table_bytes() bytes (16-byte aligned)
- * filled by linattn_rope3d_pack from fp32 DEVICE arrays cos_t, sin_t [T][pt], cos_h, sin_h [Hh][ph], cos_w, sin_w
- * [Ww][pw] (rounded to nearest fp16; the operation is defined on those fp16 values; an axis with no pairs may pass
- * NULL).  token_offset is the grid index of the call's first token: 0 for a whole clip, the first token of the
- * block for a block step (positions continue from block to block); token_offset + N may not exceed T*Hh*Ww.
- * Workspace: linattn_rope_workspace_bytes(). */
-typedef struct linattn_rope3d {
-  int32_t T, Hh, Ww;     /* latent grid */
-  int32_t pt, ph, pw;    /* feature pairs per axis */
-  const void* table;     /* DEVICE, packed by linattn_rope3d_pack (ignored by the two sizing / packing calls) */
-  int64_t token_offset;
-} linattn_rope3d;
-LINATTN_API int linattn_rope3d_table_bytes(const linattn_rope3d* rope, int32_t d, size_t* bytes);
-LINATTN_API int linattn_rope3d_pack(const linattn_rope3d* rope, int32_t d, const float* cos_t, const float* sin_t,
-                                    const float* cos_h, const float* sin_h, const float* cos_w, const float* sin_w,
-                                    void* table, void* stream);
-LINATTN_API int linattn_forward_rope3d(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v,
-                                       void* o, float eps, const linattn_rope3d* rope, void* workspace,
-                                       size_t workspace_bytes, void* stream);
-
 /* The state of Eq. 2 / Eq. 3 alone: state = (sum_n phi(k_n)^T v_n, sum_n phi(k_n)) in the layout above.
  * Deterministic: split-N partials are summed in a fixed order, so repeated calls give identical bits. */
 LINATTN_API int linattn_state(const linattn_desc* desc, int64_t N, const void* k, const void* v, float* state,
@@ -264,13 +234,6 @@ LINATTN_API int blocklin_step_rope(blocklin_cache* cache, int64_t T_b, const voi
  * q_blk and o_blk are required. */
 LINATTN_API int blocklin_peek_rope(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk,
                                    const void* v_blk, void* o_blk, const void* rope_table_blk, void* stream);
-
-/* blocklin_step_rope (commit != 0) or blocklin_peek_rope (commit = 0: the cache is only read; q_blk and o_blk
- * required) with per-axis rotary tables (see linattn_rope3d); rope->token_offset is the grid index of the block's
- * first token.  Same bits as the per-token-table calls give on the table the per-axis rotations spell out. */
-LINATTN_API int blocklin_step_rope3d(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk,
-                                     const void* v_blk, void* o_blk, const linattn_rope3d* rope, int commit,
-                                     void* stream);
 
 /* blocklin_prefill with the rotary factors: n_blocks consecutive blocks of T_b tokens over [B, n_blocks*T_b, H, d]
  * tensors, rope_table the packed rows of those n_blocks*T_b tokens; result and final cache are those of n_blocks

@@ -18,7 +18,7 @@ import os
 
 __all__ = [
     "LinAttnError", "library_path", "load_library", "state_bytes", "workspace_bytes", "new_workspace",
-    "linattn_forward", "linattn_forward_rope", "rope_pack", "Rope3D", "linattn_forward_rope3d", "new_rope_workspace", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "static_scratch_status", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
+    "linattn_forward", "linattn_forward_rope", "rope_pack", "new_rope_workspace", "linattn_state", "linattn_apply", "linattn_state_static_scratch", "static_scratch_status", "split_state", "BlockLinCache", "workspace_status", "HostForward", "kernel_launches",
     "tconv_forward", "TConvCache",
 ]
 
@@ -39,11 +39,6 @@ class LinAttnError(RuntimeError):
 class _Desc(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("d", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("stride_b", ctypes.c_int64), ("stride_n", ctypes.c_int64), ("stride_h", ctypes.c_int64)]
-
-
-class _Rope3d(ctypes.Structure):
-    _fields_ = [("T", ctypes.c_int32), ("Hh", ctypes.c_int32), ("Ww", ctypes.c_int32), ("pt", ctypes.c_int32),
-                ("ph", ctypes.c_int32), ("pw", ctypes.c_int32), ("table", ctypes.c_void_p), ("token_offset", ctypes.c_int64)]
 
 
 class _ConvDesc(ctypes.Structure):
@@ -84,10 +79,6 @@ def load_library(path: str | None = None):
         "linattn_rope_table_bytes": ([i64, ctypes.c_int32, szp], ctypes.c_int),
         "linattn_rope_pack": ([i64, ctypes.c_int32, vp, vp, vp, vp], ctypes.c_int),
         "linattn_forward_rope": ([dp, i64, vp, vp, vp, vp, f32, vp, vp, sz, vp], ctypes.c_int),
-        "linattn_rope3d_table_bytes": ([ctypes.POINTER(_Rope3d), ctypes.c_int32, szp], ctypes.c_int),
-        "linattn_rope3d_pack": ([ctypes.POINTER(_Rope3d), ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp, vp], ctypes.c_int),
-        "linattn_forward_rope3d": ([dp, i64, vp, vp, vp, vp, f32, ctypes.POINTER(_Rope3d), vp, sz, vp], ctypes.c_int),
-        "blocklin_step_rope3d": ([vp, i64, vp, vp, vp, vp, ctypes.POINTER(_Rope3d), ctypes.c_int, vp], ctypes.c_int),
         "linattn_state": ([dp, i64, vp, vp, vp, vp, sz, vp], ctypes.c_int),
         "linattn_apply": ([dp, i64, vp, vp, vp, f32, vp, sz, vp], ctypes.c_int),
         "linattn_state_static_scratch": ([dp, i64, vp, vp, vp, vp], ctypes.c_int),
@@ -252,49 +243,6 @@ def linattn_forward_rope(q, k, v, rope_table, eps: float = 1e-6, out=None, works
         workspace = new_rope_workspace(q)
     _check(lib.linattn_forward_rope(ctypes.byref(desc), N, _ptr(q), _ptr(k), _ptr(v), _ptr(o), eps, _ptr(rope_table),
                                     _ptr(workspace), workspace.numel(), _stream(q)), "linattn_forward_rope")
-    return o
-
-
-class Rope3D:
-    """Rotary factors of a T x Hh x Ww latent grid given one axis at a time (3D RoPE): three small tables instead of
-    one row per token.  ``axes``: ``((cos_t, sin_t), (cos_h, sin_h), (cos_w, sin_w))``, float32 CUDA tensors
-    ``[positions of the axis, pairs of the axis]``; pairs [0, pt) of a head follow t, the next ph follow h, the
-    rest follow w.  The packed device table is built once (by the library) and held here."""
-
-    def __init__(self, T: int, Hh: int, Ww: int, d: int, axes):
-        torch = _torch()
-        self._lib = load_library()
-        (ct, st), (ch, sh), (cw, sw) = axes
-        for n_pos, c, s_ in ((T, ct, st), (Hh, ch, sh), (Ww, cw, sw)):
-            if c.shape != s_.shape or c.dim() != 2 or c.shape[0] != n_pos or c.dtype != torch.float32 or \
-                    s_.dtype != torch.float32 or not c.is_contiguous() or not s_.is_contiguous() or not c.is_cuda:
-                raise ValueError("each axis needs contiguous float32 CUDA tensors cos, sin [positions, pairs]")
-        self.grid, self.d = (T, Hh, Ww), d
-        self.split = (ct.shape[1], ch.shape[1], cw.shape[1])
-        r = _Rope3d(T, Hh, Ww, *self.split, None, 0)
-        nb = ctypes.c_size_t()
-        _check(self._lib.linattn_rope3d_table_bytes(ctypes.byref(r), d, ctypes.byref(nb)), "linattn_rope3d_table_bytes")
-        self.table = torch.empty(nb.value, dtype=torch.uint8, device=ct.device)
-        _check(self._lib.linattn_rope3d_pack(ctypes.byref(r), d, _ptr(ct), _ptr(st), _ptr(ch), _ptr(sh), _ptr(cw), _ptr(sw),
-                                             _ptr(self.table), _stream(ct)), "linattn_rope3d_pack")
-
-    def desc(self, token_offset: int = 0) -> _Rope3d:
-        return _Rope3d(*self.grid, *self.split, self.table.data_ptr(), token_offset)
-
-
-def linattn_forward_rope3d(q, k, v, rope3d: Rope3D, eps: float = 1e-6, out=None, workspace=None, token_offset: int = 0):
-    """Eq. 2 with rotary factors given per axis of the latent grid (bf16, d = 112): the result of
-    ``linattn_forward_rope`` on the per-token table those rotations spell out, without that table."""
-    torch = _torch()
-    lib = load_library()
-    o = torch.empty_like(q) if out is None else out
-    desc = _desc_of(q, k, v, o)
-    if workspace is None:
-        workspace = new_rope_workspace(q)
-    r = rope3d.desc(token_offset)
-    _check(lib.linattn_forward_rope3d(ctypes.byref(desc), q.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o), eps,
-                                      ctypes.byref(r), _ptr(workspace), workspace.numel(), _stream(q)),
-           "linattn_forward_rope3d")
     return o
 
 
@@ -508,22 +456,6 @@ class BlockLinCache:
         o = self._rope_args(q, k, v, rope_table_blk, out, k.shape[1])
         _check(self._lib.blocklin_peek_rope(self._handle, k.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o),
                                             _ptr(rope_table_blk), _stream(k)), "blocklin_peek_rope")
-        return o
-
-    def step_rope3d(self, q, k, v, rope3d, token_offset: int, out=None, commit: bool = True):
-        """``step_rope`` (or, with commit=False, ``peek_rope``) with per-axis rotary tables (``Rope3D``);
-        token_offset: index of the block's first token in the latent grid."""
-        torch = _torch()
-        o = None
-        if q is not None:
-            o = torch.empty_like(q) if out is None else out
-            _desc_of(q, k, v, o)
-        else:
-            _desc_of(k, v)
-        self._check_layout(k)
-        r = rope3d.desc(token_offset)
-        _check(self._lib.blocklin_step_rope3d(self._handle, k.shape[1], _ptr(q), _ptr(k), _ptr(v), _ptr(o),
-                                              ctypes.byref(r), int(commit), _stream(k)), "blocklin_step_rope3d")
         return o
 
     def prefill_rope(self, q, k, v, rope_table, n_blocks: int, out=None):

@@ -101,13 +101,11 @@ size_t rope_workspace_need(const Problem& p) { return round256(rope_state_offset
 // queries (denominator from the plain ones).
 // `base` as in run_passes: the state that is added to (null: `state` itself); q may be null (state only).
 int run_rope(const Problem& p, const void* q, const void* k, const void* v, void* o, float* state, bool accumulate,
-             float eps, const __half2* rope, void* workspace, cudaStream_t stream, const float* base = nullptr,
-             const Rope3dHost* r3 = nullptr) {
+             float eps, const __half2* rope, void* workspace, cudaStream_t stream, const float* base = nullptr) {
   if (umma_rope_supported(p)) {  // one launch on the tensor cores
-    UmmaCall c{k, v, q, o, state, base, accumulate, eps, r3 ? nullptr : rope, r3};
+    UmmaCall c{k, v, q, o, state, base, accumulate, eps, rope};
     return umma_run(p, c, workspace, stream);
   }
-  if (r3) return LINATTN_ERR_UNSUPPORTED;  // per-axis tables: tensor-core path only
   if (accumulate && base && base != state) {
     if (cudaMemcpyAsync(state, base, state_bytes_of(p), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
       return LINATTN_ERR_CUDA;
@@ -196,11 +194,9 @@ static int step_impl(blocklin_cache* cache, const Problem& p, const void* q_blk,
 // One block with the rotary factors of Eq. 2.  commit: the cache takes the block (blocklin_step_rope); otherwise the
 // sum of cache and block goes to the state slot of the workspace and the cache is only read (blocklin_peek_rope).
 static int step_rope_impl(blocklin_cache* cache, const Problem& p, const void* q_blk, const void* k_blk,
-                          const void* v_blk, void* o_blk, const void* rope_table_blk, bool commit, cudaStream_t stream,
-                          const Rope3dHost* r3 = nullptr) {
+                          const void* v_blk, void* o_blk, const void* rope_table_blk, bool commit, cudaStream_t stream) {
   if (p.d & 1) return LINATTN_ERR_UNSUPPORTED;
   if ((q_blk == nullptr) != (o_blk == nullptr)) return LINATTN_ERR_INVALID_ARG;
-  if (r3) rope_table_blk = r3->table;
   if (p.N > 0 && (!k_blk || !v_blk || !rope_table_blk)) return LINATTN_ERR_INVALID_ARG;
   if (o_blk && (o_blk == q_blk || o_blk == k_blk || o_blk == v_blk)) return LINATTN_ERR_INVALID_ARG;
   int st = check_alignment(p, q_blk, k_blk, v_blk, o_blk);
@@ -212,25 +208,12 @@ static int step_rope_impl(blocklin_cache* cache, const Problem& p, const void* q
   const __half2* rope = static_cast<const __half2*>(rope_table_blk);
   if (!commit) {
     float* tmp = reinterpret_cast<float*>(static_cast<char*>(cache->workspace) + rope_state_offset(p));
-    return run_rope(p, q_blk, k_blk, v_blk, o_blk, tmp, true, cache->eps, rope, cache->workspace, stream, cache->state, r3);
+    return run_rope(p, q_blk, k_blk, v_blk, o_blk, tmp, true, cache->eps, rope, cache->workspace, stream, cache->state);
   }
-  st = run_rope(p, q_blk, k_blk, v_blk, o_blk, cache->state, true, cache->eps, rope, cache->workspace, stream, nullptr, r3);
+  st = run_rope(p, q_blk, k_blk, v_blk, o_blk, cache->state, true, cache->eps, rope, cache->workspace, stream);
   if (st != LINATTN_OK) return st;
   cache->blocks_seen += 1;
   cache->tokens_seen += p.N;
-  return LINATTN_OK;
-}
-
-// Validates a caller's per-axis rotary description for n_tokens tokens of head dim d and converts it.
-static int resolve_rope3d(const linattn_rope3d* r, const Problem& p, long long n_tokens, Rope3dHost* out) {
-  if (!r) return LINATTN_ERR_INVALID_ARG;
-  Rope3dLayout lay;
-  if (!rope3d_layout(r->T, r->Hh, r->Ww, r->pt, r->ph, r->pw, p.d, &lay)) return LINATTN_ERR_UNSUPPORTED;
-  if (!umma_rope_supported(p)) return LINATTN_ERR_UNSUPPORTED;
-  if (r->token_offset < 0 || r->token_offset + n_tokens > (long long)r->T * r->Hh * r->Ww) return LINATTN_ERR_INVALID_ARG;
-  if (n_tokens > 0 && !r->table) return LINATTN_ERR_INVALID_ARG;
-  if (!aligned16(r->table)) return LINATTN_ERR_BAD_ALIGNMENT;
-  *out = Rope3dHost{r->T, r->Hh, r->Ww, r->pt, r->ph, r->pw, r->table, r->token_offset};
   return LINATTN_OK;
 }
 
@@ -391,44 +374,6 @@ int linattn_forward_rope(const linattn_desc* desc, int64_t N, const void* q, con
   if (N == 0) return LINATTN_OK;
   float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + rope_state_offset(p));
   return run_rope(p, q, k, v, o, state, false, eps, static_cast<const __half2*>(rope_table), workspace, (cudaStream_t)stream);
-}
-
-int linattn_rope3d_table_bytes(const linattn_rope3d* rope, int32_t d, size_t* bytes) {
-  if (!rope || !bytes) return LINATTN_ERR_INVALID_ARG;
-  Rope3dLayout lay;
-  if (!rope3d_layout(rope->T, rope->Hh, rope->Ww, rope->pt, rope->ph, rope->pw, d, &lay)) return LINATTN_ERR_UNSUPPORTED;
-  *bytes = lay.bytes;
-  return LINATTN_OK;
-}
-
-int linattn_rope3d_pack(const linattn_rope3d* rope, int32_t d, const float* cos_t, const float* sin_t, const float* cos_h,
-                        const float* sin_h, const float* cos_w, const float* sin_w, void* table, void* stream) {
-  if (!rope || !table) return LINATTN_ERR_INVALID_ARG;
-  Rope3dLayout lay;
-  if (!rope3d_layout(rope->T, rope->Hh, rope->Ww, rope->pt, rope->ph, rope->pw, d, &lay)) return LINATTN_ERR_UNSUPPORTED;
-  if (!aligned16(table)) return LINATTN_ERR_BAD_ALIGNMENT;
-  const float* cs[3] = {cos_t, cos_h, cos_w};
-  const float* sn[3] = {sin_t, sin_h, sin_w};
-  for (int a = 0; a < 3; ++a)
-    if (lay.count[a] > 0 && (!cs[a] || !sn[a])) return LINATTN_ERR_INVALID_ARG;
-  return cuda_status(rope3d_pack(lay, cs, sn, table, (cudaStream_t)stream));
-}
-
-int linattn_forward_rope3d(const linattn_desc* desc, int64_t N, const void* q, const void* k, const void* v, void* o,
-                           float eps, const linattn_rope3d* rope, void* workspace, size_t workspace_bytes, void* stream) {
-  Problem p;
-  int st = resolve(desc, N, &p);
-  if (st != LINATTN_OK) return st;
-  if (!workspace) return LINATTN_ERR_INVALID_ARG;
-  Rope3dHost r3;
-  if ((st = resolve_rope3d(rope, p, N, &r3)) != LINATTN_OK) return st;
-  if (N > 0 && (!q || !k || !v || !o || o == q || o == k || o == v)) return LINATTN_ERR_INVALID_ARG;
-  if ((st = check_alignment(p, q, k, v, o)) != LINATTN_OK) return st;
-  if (!aligned16(workspace)) return LINATTN_ERR_BAD_ALIGNMENT;
-  if (workspace_bytes < rope_workspace_need(p)) return LINATTN_ERR_WORKSPACE_TOO_SMALL;
-  if (N == 0) return LINATTN_OK;
-  float* state = reinterpret_cast<float*>(static_cast<char*>(workspace) + rope_state_offset(p));
-  return run_rope(p, q, k, v, o, state, false, eps, nullptr, workspace, (cudaStream_t)stream, nullptr, &r3);
 }
 
 uint64_t linattn_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
@@ -593,18 +538,6 @@ int blocklin_peek_rope(blocklin_cache* cache, int64_t T_b, const void* q_blk, co
   if (st != LINATTN_OK) return st;
   if (p.N > 0 && (!q_blk || !o_blk)) return LINATTN_ERR_INVALID_ARG;
   return step_rope_impl(cache, p, q_blk, k_blk, v_blk, o_blk, rope_table_blk, false, (cudaStream_t)stream);
-}
-
-int blocklin_step_rope3d(blocklin_cache* cache, int64_t T_b, const void* q_blk, const void* k_blk, const void* v_blk,
-                         void* o_blk, const linattn_rope3d* rope, int commit, void* stream) {
-  if (!cache || cache->magic != kCacheMagic) return LINATTN_ERR_BAD_HANDLE;
-  Problem p;
-  int st = resolve(&cache->desc, T_b, &p);
-  if (st != LINATTN_OK) return st;
-  Rope3dHost r3;
-  if ((st = resolve_rope3d(rope, p, T_b, &r3)) != LINATTN_OK) return st;
-  if (!commit && p.N > 0 && (!q_blk || !o_blk)) return LINATTN_ERR_INVALID_ARG;
-  return step_rope_impl(cache, p, q_blk, k_blk, v_blk, o_blk, nullptr, commit != 0, (cudaStream_t)stream, &r3);
 }
 
 int blocklin_prefill_rope(blocklin_cache* cache, int64_t n_blocks, int64_t T_b, const void* q, const void* k,

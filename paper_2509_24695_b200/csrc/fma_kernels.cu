@@ -288,47 +288,7 @@ __global__ void prefix_states_kernel(float4* __restrict__ blk, float4* __restric
   cache[b * per_batch4 + e] = run;
 }
 
-// Packed per-axis rotary table: one thread per (cos, sin) slot.  A slot whose pair lies outside its axis' range holds
-// the identity rotation.
-struct Rope3dPackArgs {
-  const float* cs[3];
-  const float* sn[3];
-  unsigned base[3], nch[3], clo[3], start[3], count[3], positions[3];
-};
-__global__ void rope3d_pack_kernel(Rope3dPackArgs a, unsigned total, __half2* __restrict__ out) {
-  const unsigned i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= total) return;
-  int axis = 2;
-  if (i < a.base[1] / 4) axis = 0;
-  else if (i < a.base[2] / 4) axis = 1;
-  const unsigned local = i - a.base[axis] / 4;                 // slot within the axis' sub-table
-  const unsigned per_pos = a.nch[axis] * 4;
-  const unsigned pos = local / per_pos, pair = a.clo[axis] * 4 + local % per_pos;
-  __half2 v = __floats2half2_rn(1.f, 0.f);
-  if (pair >= a.start[axis] && pair < a.start[axis] + a.count[axis]) {
-    const size_t src = (size_t)pos * a.count[axis] + (pair - a.start[axis]);
-    v = __floats2half2_rn(a.cs[axis][src], a.sn[axis][src]);
-  }
-  out[i] = v;
-}
-
 }  // namespace
-
-cudaError_t rope3d_pack(const Rope3dLayout& lay, const float* const cs[3], const float* const sn[3], void* table,
-                        cudaStream_t stream) {
-  Rope3dPackArgs a;
-  unsigned total = 0;
-  for (int x = 0; x < 3; ++x) {
-    a.cs[x] = cs[x]; a.sn[x] = sn[x];
-    a.base[x] = lay.base[x]; a.nch[x] = lay.nch[x]; a.clo[x] = lay.clo[x];
-    a.start[x] = lay.start[x]; a.count[x] = lay.count[x]; a.positions[x] = lay.positions[x];
-    total += lay.positions[x] * lay.nch[x] * 4;
-  }
-  if (total == 0) return cudaSuccess;
-  rope3d_pack_kernel<<<(total + 255) / 256, 256, 0, stream>>>(a, total, static_cast<__half2*>(table));
-  count_launches(1);
-  return cudaGetLastError();
-}
 
 cudaError_t prefix_states(float* blk, float* cache, int B, int M, long long floats_per_batch, cudaStream_t stream) {
   const long long n4 = floats_per_batch / 4;

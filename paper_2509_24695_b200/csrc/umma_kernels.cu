@@ -178,74 +178,6 @@ struct TileWalk {
   __device__ void next() { ++f; if (++tp == w.mm) { tp = 0; ++uo; } }
 };
 
-// Rotary factors that depend on a token's (frame, row, column) position one axis at a time (3D RoPE): instead of a
-// table row per token, one small table per axis.  Feature pairs [0, s1) turn with the frame index, [s1, s2) with the
-// row, the rest with the column.  Axis a's sub-table holds, per position, the 16-byte chunks (four (cos, sin) fp16
-// pairs) that touch its pair range, with the identity rotation at pairs that belong to a neighbouring axis.  The
-// whole thing is a few KB and stays in L1, where a per-token table costs as many bytes from L2 as Q or K themselves.
-struct Rope3dDev {
-  const uint8_t* table;
-  unsigned HW, Ww, Hh;               // Hh * Ww, columns, rows of the latent grid (tokens frame-major, then row, then column)
-  unsigned base[3], nch[3], clo[3];  // per axis: byte offset of its sub-table, chunks per position, first chunk
-  unsigned s1, s2;
-  unsigned n_off;                    // grid index of the call's first token
-};
-
-// Where one thread finds its 16-byte chunk column (four pairs): at most two axes meet in a chunk.
-// meta: row pitch of axis 1's sub-table | pitch 2 << 8 | axis 1 << 16 | axis 2 << 18 | pairs taken from axis 2 << 20
-struct ChunkSrc { unsigned off1, off2, meta; };
-
-__device__ __forceinline__ ChunkSrc chunk_src(const Rope3dDev& r, int c) {
-  auto axis_of = [&](unsigned pair) { return pair < r.s1 ? 0u : pair < r.s2 ? 1u : 2u; };
-  const unsigned a1 = axis_of(4u * c), a2 = axis_of(4u * c + 3u);
-  unsigned mask = 0;
-  for (unsigned j = 0; j < 4; ++j)
-    if (a2 != a1 && axis_of(4u * c + j) == a2) mask |= 1u << j;
-  ChunkSrc s;
-  s.off1 = r.base[a1] + ((unsigned)c - r.clo[a1]) * 16u;
-  s.off2 = r.base[a2] + ((unsigned)c - r.clo[a2]) * 16u;
-  s.meta = (r.nch[a1] * 16u) | ((r.nch[a2] * 16u) << 8) | (a1 << 16) | (a2 << 18) | (mask << 20);
-  return s;
-}
-
-// A thread's place in the latent grid.  Its rows come in ascending order with small steps (32 tokens) except at the
-// start of a segment, so the position is advanced with carries and only re-derived by division after a jump.
-struct RotCursor { unsigned n, t, h, w; };
-
-__device__ __forceinline__ void rot_seek(const Rope3dDev& r, RotCursor& c, unsigned n) {
-  const unsigned delta = n - c.n;
-  if (delta < 1024u) {
-    c.w += delta;
-    while (c.w >= r.Ww) {
-      c.w -= r.Ww;
-      if (++c.h == r.Hh) { c.h = 0; ++c.t; }
-    }
-  } else {
-    c.t = n / r.HW;
-    const unsigned rem = n - c.t * r.HW;
-    c.h = rem / r.Ww;
-    c.w = rem - c.h * r.Ww;
-  }
-  c.n = n;
-}
-
-__device__ __forceinline__ uint4 rot3d_load(const Rope3dDev& r, const ChunkSrc& s, const RotCursor& c) {
-  const unsigned a1 = (s.meta >> 16) & 3u;
-  const unsigned p1 = a1 == 0 ? c.t : a1 == 1 ? c.h : c.w;
-  uint4 e = __ldg(reinterpret_cast<const uint4*>(r.table + s.off1 + p1 * (s.meta & 0xFFu)));
-  const unsigned mask = s.meta >> 20;
-  if (mask) {   // a chunk where two axes meet: the later pairs come from the second axis' table
-    const unsigned a2 = (s.meta >> 18) & 3u;
-    const unsigned p2 = a2 == 1 ? c.h : c.w;
-    const uint4 f = __ldg(reinterpret_cast<const uint4*>(r.table + s.off2 + p2 * ((s.meta >> 8) & 0xFFu)));
-    if (mask & 1u) e.x = f.x;
-    if (mask & 2u) e.y = f.y;
-    if (mask & 4u) e.z = f.z;
-    if (mask & 8u) e.w = f.w;
-  }
-  return e;
-}
-
 struct FusedParams {
   int B, H, HG;            // HG: head groups per batch entry = ceil(H / G)
   Sched sa, sc;            // state pass (64-token stages) and apply pass (128-token tiles)
@@ -259,7 +191,6 @@ struct FusedParams {
   uint8_t* s_image;        // non-null: the reduce also leaves every unit's S operand (bf16 hi + lo, in the shared-memory
                            // layout) here, S_BYTES per unit, and the apply pass fetches it with one bulk copy
   const uint4* rope;       // rotary variant: [N][d/8] chunks of four (cos, sin) fp16 pairs; null otherwise
-  Rope3dDev r3;            // rotary variant with per-axis tables (R3D instantiation)
   long long N;             // tokens (bound of the rotary table)
 };
 
@@ -719,7 +650,7 @@ __device__ __forceinline__ void build_s_operand(uint8_t* s_op, const float* __re
 }
 
 // ============================================================================ the kernel
-template <int D, bool ROPE, bool R3D>
+template <int D, bool ROPE>
 __global__ void __launch_bounds__(Roles<ROPE>::THREADS, 1)
 umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                   const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o, FusedParams p) {
@@ -887,22 +818,13 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     // Of the second K box these warps take the first 32 token rows of a stage; the epilogue warps, idle until the
     // segment's accumulators are complete, take the other 32 (this role is what the pass waits for).
     uint4 tab0[kTileState / 32], tab1[1];
-    RotCursor cur = {0u, 0u, 0u, 0u};
-    ChunkSrc src0 = {0u, 0u, 0u}, src1 = {0u, 0u, 0u};
-    if (ROPE && R3D) { src0 = chunk_src(p.r3, lc); if (box1_live) src1 = chunk_src(p.r3, 8 + lc); }
     auto fetch_rot = [&](int tile, int i) {
       const long long n = (long long)tile * kTileState + row0 + 32 * i;
       tab0[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
       if (i == 0) tab1[0] = tab0[i];
       if (n < p.N) {
-        if (R3D) {
-          rot_seek(p.r3, cur, (unsigned)n + p.r3.n_off);
-          tab0[i] = rot3d_load(p.r3, src0, cur);
-          if (i == 0 && box1_live) tab1[0] = rot3d_load(p.r3, src1, cur);
-        } else {
-          tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
-          if (i == 0 && box1_live) tab1[0] = __ldg(p.rope + n * (D / 8) + 8 + lc);
-        }
+        tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
+        if (i == 0 && box1_live) tab1[0] = __ldg(p.rope + n * (D / 8) + 8 + lc);
       }
     };
     if (ROPE) {
@@ -990,20 +912,10 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 #pragma unroll
     for (int e = 0; e < 4; ++e) zh[e] = make_float2(0.f, 0.f);
     uint4 tabh[2];
-    RotCursor curh = {0u, 0u, 0u, 0u};
-    ChunkSrc srch = {0u, 0u, 0u};
-    if (ROPE && R3D && h_live) srch = chunk_src(p.r3, 8 + lch);
     auto fetch_roth = [&](int tile, int j) {
       const long long n = (long long)tile * kTileState + 32 + row0h + 16 * j;
       tabh[j] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
-      if (h_live && n < p.N) {
-        if (R3D) {
-          rot_seek(p.r3, curh, (unsigned)n + p.r3.n_off);
-          tabh[j] = rot3d_load(p.r3, srch, curh);
-        } else {
-          tabh[j] = __ldg(p.rope + n * (D / 8) + 8 + lch);
-        }
-      }
+      if (h_live && n < p.N) tabh[j] = __ldg(p.rope + n * (D / 8) + 8 + lch);
     };
     if (ROPE) {
       TileWalk t0(wa);
@@ -1187,21 +1099,12 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     for (int e = 0; e < 8; ++e) zc[e] = make_float2(0.f, 0.f);
     // rotations one tile ahead, as in the state pass
     uint4 tab0[kTileApply / 32], tab1[kTileApply / 32];
-    RotCursor cur = {0u, 0u, 0u, 0u};
-    ChunkSrc src0 = {0u, 0u, 0u}, src1 = {0u, 0u, 0u};
-    if (ROPE && R3D) { src0 = chunk_src(p.r3, lc); if (box1_live) src1 = chunk_src(p.r3, 8 + lc); }
     auto fetch_rot = [&](int tile, int i) {
       const long long n = (long long)tile * kTileApply + row0 + 32 * i;
       tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
       if (n < p.N) {
-        if (R3D) {
-          rot_seek(p.r3, cur, (unsigned)n + p.r3.n_off);
-          tab0[i] = rot3d_load(p.r3, src0, cur);
-          if (box1_live) tab1[i] = rot3d_load(p.r3, src1, cur);
-        } else {
-          tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
-          if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
-        }
+        tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
+        if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
       }
     };
     if (ROPE) {
@@ -1457,7 +1360,7 @@ int sm_count() {
 
 inline int groups_of(int d) { return d == 32 ? 4 : d == 64 ? 2 : 1; }
 
-template <int D, bool ROPE, bool R3D = false>
+template <int D, bool ROPE>
 int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
   using C = Cfg<D>;
   const int sms = sm_count();
@@ -1474,16 +1377,6 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   fp.eps = c.eps;
   fp.ctrl = static_cast<WorkspaceCtrl*>(workspace);
   fp.rope = static_cast<const uint4*>(c.rope);
-  if (R3D) {
-    const Rope3dHost& h = *c.rope3d;
-    Rope3dLayout lay;
-    if (!rope3d_layout(h.T, h.Hh, h.Ww, h.pt, h.ph, h.pw, p.d, &lay)) return LINATTN_ERR_UNSUPPORTED;
-    fp.r3.table = static_cast<const uint8_t*>(h.table);
-    fp.r3.HW = (unsigned)(h.Hh * h.Ww); fp.r3.Ww = (unsigned)h.Ww; fp.r3.Hh = (unsigned)h.Hh;
-    for (int a = 0; a < 3; ++a) { fp.r3.base[a] = lay.base[a]; fp.r3.nch[a] = lay.nch[a]; fp.r3.clo[a] = lay.clo[a]; }
-    fp.r3.s1 = (unsigned)h.pt; fp.r3.s2 = (unsigned)(h.pt + h.ph);
-    fp.r3.n_off = (unsigned)h.token_offset;
-  }
   fp.N = p.N;
   fp.s_image = nullptr;
   if (do_state && do_apply && C::G == 1 && fp.sa.P >= 1) {
@@ -1520,13 +1413,13 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LINATTN_ERR_CUDA;
   if (!attr_set[dev]) {
-    if (cudaFuncSetAttribute(umma_fused_kernel<D, ROPE, R3D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM) !=
+    if (cudaFuncSetAttribute(umma_fused_kernel<D, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM) !=
         cudaSuccess)
       return LINATTN_ERR_CUDA;
     attr_set[dev] = true;
   }
   void* args[] = {&mk, &mv, &mq, &mo, &fp};
-  const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D, ROPE, R3D>, dim3(grid), dim3(Roles<ROPE>::THREADS), args,
+  const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D, ROPE>, dim3(grid), dim3(Roles<ROPE>::THREADS), args,
                                                     C::SMEM, stream);
   if (e != cudaSuccess) { cudaGetLastError(); return LINATTN_ERR_CUDA; }
   count_launches(1);
@@ -1555,12 +1448,10 @@ bool umma_rope_supported(const Problem& p) { return umma_supported(p) && p.d == 
 int umma_run(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
   if (p.N == 0 || (!c.k && !c.q)) return LINATTN_OK;
   switch (p.d) {
-    case 32: return (c.rope || c.rope3d) ? LINATTN_ERR_UNSUPPORTED : launch_fused<32, false>(p, c, workspace, stream);
-    case 64: return (c.rope || c.rope3d) ? LINATTN_ERR_UNSUPPORTED : launch_fused<64, false>(p, c, workspace, stream);
-    case 112:
-      if (c.rope3d) return launch_fused<112, true, true>(p, c, workspace, stream);
-      return c.rope ? launch_fused<112, true>(p, c, workspace, stream) : launch_fused<112, false>(p, c, workspace, stream);
-    case 128: return (c.rope || c.rope3d) ? LINATTN_ERR_UNSUPPORTED : launch_fused<128, false>(p, c, workspace, stream);
+    case 32: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<32, false>(p, c, workspace, stream);
+    case 64: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<64, false>(p, c, workspace, stream);
+    case 112: return c.rope ? launch_fused<112, true>(p, c, workspace, stream) : launch_fused<112, false>(p, c, workspace, stream);
+    case 128: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<128, false>(p, c, workspace, stream);
   }
   return LINATTN_ERR_UNSUPPORTED;
 }

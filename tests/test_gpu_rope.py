@@ -190,90 +190,3 @@ def test_rope_prefill_equals_steps_and_oracle(la, orc, case):
     cache.reset()
     assert cache.prefill_rope(None, kd, vd, table, M) is None        # context only
     assert torch.equal(cache.state, final) and cache.status() == 0
-
-
-def axes_on_device(la, T, Hh, Ww, d, split=None):
-    (ct, st), (ch, sh), (cw, sw), split = synth.rope_axes(T, Hh, Ww, d, split=split)
-    r3 = la.Rope3D(T, Hh, Ww, d, ((to_dev(ct), to_dev(st)), (to_dev(ch), to_dev(sh)), (to_dev(cw), to_dev(sw))))
-    assert r3.split == split
-    cos, sin = synth.rope_table(T, Hh, Ww, d, split=split)       # the same rotations spelled out per token
-    table = la.rope_pack(to_dev(cos), to_dev(sin))
-    packed = table.cpu().numpy().astype(np.float64)
-    return r3, table, packed[..., 0], packed[..., 1]
-
-
-# grid (T, Hh, Ww), heads, batch, split of the 56 pairs over (t, h, w): the default split 20/18/18 has a group of four
-# pairs where the h and w axes meet; 24/16/16 has none; 22/17/17 has two; 0/28/28 and 56/0/0 leave axes empty
-ROPE3D_CASES = [((5, 10, 20), 3, 2, None), ((3, 7, 9), 20, 1, (24, 16, 16)), ((2, 3, 129), 2, 1, (22, 17, 17)),
-                ((4, 6, 5), 5, 2, (0, 28, 28)), ((9, 1, 1), 2, 1, (56, 0, 0)), ((1, 1, 1), 1, 1, None),
-                ((2, 30, 52), 20, 1, None)]
-
-
-@pytest.mark.parametrize("case", ROPE3D_CASES, ids=lambda c: "T%dx%dx%d_H%d_B%d_%s" % (*c[0], c[1], c[2], "def" if c[3] is None else "%d_%d_%d" % c[3]))
-def test_rope3d_forward_equals_the_per_token_table_and_the_oracle(la, orc, case):
-    """Per-axis rotary tables (3D RoPE, Sec. 3.1): the same bits as the per-token-table path on the table those
-    rotations spell out, and the oracle's Eq. 2 with rotary factors on that table."""
-    import torch
-
-    (T, Hh, Ww), H, B, split = case
-    N, d = T * Hh * Ww, 112
-    q, k, v = gen(B, N, H, d, 5700 + N, "bf16")
-    r3, table, cs, sn = axes_on_device(la, T, Hh, Ww, d, split)
-    qd, kd, vd = to_dev(q), to_dev(k), to_dev(v)
-    o3 = la.linattn_forward_rope3d(qd, kd, vd, r3, EPS)
-    o1 = la.linattn_forward_rope(qd, kd, vd, table, EPS)
-    assert torch.equal(o3, o1)
-    assert_parity_bf16(to_f64(o3), orc.rope_forward(q, k, v, cs, sn, EPS), f"rope3d forward {case}")
-
-
-def test_rope3d_block_steps_peek_and_offsets(la, orc):
-    """Cached steps with per-axis tables: blocks of whole frames and a ragged last block, read-only steps, the bits of
-    the per-token-table steps, the oracle's block-causal rotary form."""
-    import torch
-
-    (T, Hh, Ww), H, B, d = (7, 6, 10), 3, 2, 112
-    N, T_b = T * Hh * Ww, 2 * Hh * Ww + 7                     # blocks that do not end on frame boundaries
-    q, k, v = gen(B, N, H, d, 5800, "bf16")
-    r3, table, cs, sn = axes_on_device(la, T, Hh, Ww, d)
-    c3 = la.BlockLinCache(B, H, d, torch.bfloat16, "cuda", max_T_b=T_b, eps=EPS)
-    c1 = la.BlockLinCache(B, H, d, torch.bfloat16, "cuda", max_T_b=T_b, eps=EPS)
-    outs = []
-    for n0 in range(0, N, T_b):
-        sl = slice(n0, min(n0 + T_b, N))
-        blk = [to_dev(np.ascontiguousarray(x[:, sl])) for x in (q, k, v)]
-        before = c3.state.clone()
-        peek = c3.step_rope3d(*blk, r3, n0, commit=False)
-        assert torch.equal(c3.state, before) and c3.info()["blocks_seen"] == n0 // T_b
-        o3 = c3.step_rope3d(*blk, r3, n0)
-        o1 = c1.step_rope(*blk, table[sl].contiguous())
-        assert torch.equal(peek, o3) and torch.equal(o3, o1) and torch.equal(c3.state, c1.state)
-        outs.append(o3)
-    assert_parity_bf16(to_f64(torch.cat(outs, dim=1)), orc.rope_forward(q, k, v, cs, sn, EPS, T_b=T_b), "rope3d steps")
-    # absorb only, then the same cache
-    c4 = la.BlockLinCache(B, H, d, torch.bfloat16, "cuda", max_T_b=N, eps=EPS)
-    assert c4.step_rope3d(None, to_dev(k), to_dev(v), r3, 0) is None and c4.status() == 0
-
-
-def test_rope3d_errors(la):
-    import torch
-
-    one = lambda n, p: (torch.ones((n, p), device="cuda"), torch.zeros((n, p), device="cuda"))
-    r3 = la.Rope3D(2, 3, 4, 112, (one(2, 20), one(3, 18), one(4, 18)))
-    x = torch.zeros((1, 24, 2, 112), dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(la.LinAttnError) as e:      # more tokens than the grid has
-        la.linattn_forward_rope3d(torch.zeros((1, 25, 2, 112), dtype=torch.bfloat16, device="cuda"), *(torch.zeros((1, 25, 2, 112), dtype=torch.bfloat16, device="cuda") for _ in range(2)), r3, EPS)
-    assert e.value.status == -1
-    with pytest.raises(la.LinAttnError) as e:      # the offset pushes the call past the grid's end
-        la.linattn_forward_rope3d(x, x.clone(), x.clone(), r3, EPS, token_offset=1)
-    assert e.value.status == -1
-    with pytest.raises(la.LinAttnError) as e:      # three axes inside one group of four pairs
-        la.Rope3D(2, 3, 4, 112, (one(2, 21), one(3, 2), one(4, 33)))
-    assert e.value.status == -2
-    with pytest.raises(la.LinAttnError) as e:      # pairs do not add up to d/2
-        la.Rope3D(2, 3, 4, 112, (one(2, 20), one(3, 18), one(4, 17)))
-    assert e.value.status == -2
-    x64 = torch.zeros((1, 24, 2, 64), dtype=torch.bfloat16, device="cuda")
-    r64 = la.Rope3D(2, 3, 4, 64, (one(2, 12), one(3, 10), one(4, 10)))
-    with pytest.raises(la.LinAttnError) as e:      # the per-axis form runs on the tensor-core path of d = 112 only
-        la.linattn_forward_rope3d(x64, x64.clone(), x64.clone(), r64, EPS)
-    assert e.value.status == -2
