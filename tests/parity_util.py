@@ -20,8 +20,11 @@ def to_f64(t):
     return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
 
 
-def assert_parity_bf16(got, ref, what=""):
+def assert_parity_bf16(got, ref, what="", rms_rel=1e-2):
     """bf16 I/O with fp32 accumulation.  `got`, `ref`: float64 [B, n, H, d].
+    rms_rel: weight of the head's RMS in bar 2 (1e-2; the rotary tensor-core path, which also rounds the rotated
+    queries and keys to bf16, is given 1.5e-2 where hundreds of thousands of elements are compared: its per-element
+    error has a standard deviation of about 0.2 % of the RMS, and the largest of 6e5 samples reaches five of them).
 
     1. the stated bar: |delta| <= 1e-2 + 1e-2*|ref| per element;
     2. the same with the absolute term scaled by the head's RMS of ref, because with zero-mean V the
@@ -33,9 +36,9 @@ def assert_parity_bf16(got, ref, what=""):
     delta = np.abs(got - ref)
     assert (delta <= 1e-2 + 1e-2 * np.abs(ref)).all(), f"{what}: stated tolerance, max delta {delta.max():.3e}"
     rms = np.sqrt((ref ** 2).mean(axis=(1, 3), keepdims=True))
-    bad = delta > 1e-2 * rms + 1e-2 * np.abs(ref)
+    bad = delta > rms_rel * rms + 1e-2 * np.abs(ref)
     assert not bad.any(), (f"{what}: RMS-scaled tolerance: {bad.sum()} of {bad.size} elements, "
-                           f"worst ratio {(delta / (1e-2 * rms + 1e-2 * np.abs(ref) + 1e-300)).max():.3f}")
+                           f"worst ratio {(delta / (rms_rel * rms + 1e-2 * np.abs(ref) + 1e-300)).max():.3f}")
     num = np.sqrt((delta ** 2).sum(axis=(1, 3)))
     den = np.sqrt((ref ** 2).sum(axis=(1, 3)))
     ok = num <= 5e-3 * den + 1e-300
