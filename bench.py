@@ -388,7 +388,7 @@ def main():
         if not args.no_extras:
             ex = extras(torch, la, synth, dev, peak)
             out["other_workloads"] = ex
-            # the figures the path is judged on, in one compact place: every hot-path workload against the measured
+            # every hot-path workload in one compact place, each against the measured
             # copy peak ("frac") and against the nominal 8 TB/s ("frac_8tbs")
             pw = {w.name + "_forward": frac_entry(ms_per_step * 1e3, kern["forward"]["bytes"], peak),
                   w.name + "_state_alone": frac_entry(ms_state * 1e3, kern["state"]["bytes"], peak),
