@@ -83,7 +83,7 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, 
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// ---------------------------------------------------------------- TMA (tiled, 4-D, no multicast)
+// ---------------------------------------------------------------- TMA (tiled, 4-D; every load lands in this CTA alone)
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
