@@ -34,6 +34,8 @@ if ROOT not in sys.path:
 # dram__bytes_read.sum + dram__bytes_write.sum per forward launch, from the ncu capture summarised under
 # profiles/ (None once the kernel has changed since the counters were taken)
 NCU_TRAFFIC_BYTES = {"480p_5s_bidir": 556.3e6}
+# the same for side workloads whose dominant launch was captured (keys of roofline.per_workload)
+NCU_TRAFFIC_SIDE = {"720p_minute_stream_step": 362.9e6, "480p_5s_bidir_rope": 573.8e6}
 
 METRIC = "linear_attn_tokens_heads_per_s"
 UNIT = "tokens*heads/s"
@@ -404,6 +406,9 @@ def main():
                     pw[name] = frac_entry(e["ms"] * 1e3, e["algorithmic_gbs"] * e["ms"] * 1e6, peak)
                 elif "step_latency_us" in e and "algorithmic_gbs" in e:
                     pw[name] = frac_entry(e["step_latency_us"], e["algorithmic_gbs"] * e["step_latency_us"] * 1e3, peak)
+            for name, traffic in NCU_TRAFFIC_SIDE.items():
+                if name in pw:
+                    pw[name]["traffic"] = traffic
             roofline["per_workload"] = pw
     if rank == 0:
         print(json.dumps(out))
