@@ -94,7 +94,9 @@ struct Cfg {
   // per SM the memory system's queues grow and the SMs' shares of the bandwidth drift apart.
   static constexpr int STATE_STAGES = DATA_BYTES / STAGE_BYTES < 4 ? DATA_BYTES / STAGE_BYTES : 4;
   static constexpr int BAR_BYTES = 1024;
-  static constexpr size_t SMEM = 1024 + DATA_BYTES + BAR_BYTES;
+  // rotary variant without row padding (d = 128): the denominators of a tile's rows travel in a small array per slot
+  static constexpr int DEN_BYTES = D == 128 ? APPLY_SLOTS * kTileApply * 4 : 0;
+  static constexpr size_t SMEM = 1024 + DATA_BYTES + BAR_BYTES + DEN_BYTES;
 };
 
 // How the (unit, token tile) work of one pass is dealt to the persistent grid.
@@ -520,8 +522,9 @@ __device__ __forceinline__ void reduce_image_zrow(const FusedParams& p, int u, i
   using C = Cfg<D>;
   constexpr int E4 = (D + 1) * D / 4, REC4 = E4 + kZParts / 4, Z4 = D / 4, NR = 6;
   static_assert((16 * Z4) % 32 == 0 && Z4 % 2 == 0, "whole warps take part in the shuffles");
-  const int t = (int)threadIdx.x;
-  if (t >= 16 * Z4) return;
+  // sixteen threads per float4 of z; with fewer than 16 * Z4 threads (d = 128: 512 wanted, 480 there) the first warps
+  // take a second turn (whole warps: the shuffles below stay inside a warp)
+  for (int t = (int)threadIdx.x; t < 16 * Z4; t += ((int)blockDim.x / 32) * 32) {
   const int hc = t >> 4, w = t & 15;
   const Sched& s = p.sa;
   auto record_of = [&](int kk) { return kk < ncol ? kk * s.U + u : s.P * s.U + r_lo + (kk - ncol) + u; };
@@ -551,9 +554,9 @@ __device__ __forceinline__ void reduce_image_zrow(const FusedParams& p, int u, i
   float4 up;   // the upper half of this chunk, from the lane that holds float4 hc + 1
   up.x = __shfl_xor_sync(0xffffffffu, sum.x, 16); up.y = __shfl_xor_sync(0xffffffffu, sum.y, 16);
   up.z = __shfl_xor_sync(0xffffffffu, sum.z, 16); up.w = __shfl_xor_sync(0xffffffffu, sum.w, 16);
-  if (w != 0) return;
+  if (w != 0) continue;
   reinterpret_cast<float4*>(p.state)[e4] = sum;
-  if (hc & 1) return;
+  if (hc & 1) continue;
   const float x[8] = {sum.x, sum.y, sum.z, sum.w, up.x, up.y, up.z, up.w};
   uint32_t hi[4], lo[4];
 #pragma unroll
@@ -567,6 +570,7 @@ __device__ __forceinline__ void reduce_image_zrow(const FusedParams& p, int u, i
   uint8_t* img = p.s_image + (size_t)u * C::S_BYTES;
   *reinterpret_cast<uint4*>(img + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
   *reinterpret_cast<uint4*>(img + 2 * C::SBOX_BYTES + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
 }
 
 template <int D, bool ROPE>
@@ -686,6 +690,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   uint64_t* seg_done = s_ready + 1;        // every MMA of the finished segment is complete
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(seg_done + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  float* den_rows = reinterpret_cast<float*>(smem + C::DATA_BYTES + C::BAR_BYTES);   // [NSC][128], d = 128 with rotary factors
   static_assert((3 * NSA + 5 + 4 * NSC + 6) * 8 + 8 <= C::BAR_BYTES, "barrier block too small");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1004,7 +1009,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
           }
         }
       }
-      if (C::ONES_BOX) {
+      if (C::ONES_BOX && !ROPE) {   // (rotary: z comes from the ReLU warps)
         float zsum = 0.f;
 #pragma unroll 1
         for (int a = 0; a < C::STATE_ACCS; ++a) {
@@ -1176,7 +1181,11 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
           den += __shfl_xor_sync(0xffffffffu, den, 1);
           den += __shfl_xor_sync(0xffffffffu, den, 2);
           den += __shfl_xor_sync(0xffffffffu, den, 4);
-          if (lc == 6) *reinterpret_cast<float*>(c1) = den;  // chunk 6 of the second box: features 112..119
+          if (D == 112) {
+            if (lc == 6) *reinterpret_cast<float*>(c1) = den;  // chunk 6 of the second box: features 112..119
+          } else {
+            if (pc == 0) den_rows[s * kTileApply + row0 + 32 * i] = den;   // no padding to carry it
+          }
         }
         fence_proxy_async_smem();
         mbar_arrive(&c_ready[s]);
@@ -1215,7 +1224,8 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       float rinv[C::G];
       if (ROPE) {
         // the ReLU warps left phi(q) . z of this row in the row's padding
-        const float den = *reinterpret_cast<const float*>(sl + HALF + r * kRowBytes + ((6 ^ (r & 7)) << 4));
+        const float den = D == 112 ? *reinterpret_cast<const float*>(sl + HALF + r * kRowBytes + ((6 ^ (r & 7)) << 4))
+                                   : den_rows[s * kTileApply + r];
         rinv[0] = 1.0f / (den + p.eps);
       } else {
         uint32_t dn[4];
@@ -1441,9 +1451,10 @@ size_t umma_partial_bytes(const Problem& p, bool rope) {
   return ((size_t)kMaxCtas + units) * (G * (size_t)p.state_elems() + (rope ? kZParts : 0)) * sizeof(float);
 }
 
-// The rotary variant runs on the tensor cores at the paper's head dim (the denominators travel in the zero
-// padding of the 112-feature rows); other shapes take the FMA kernels.
-bool umma_rope_supported(const Problem& p) { return umma_supported(p) && p.d == 112; }
+// The rotary variant runs on the tensor cores at the one-head-per-operand head dims: 112, the paper's (the
+// denominators travel in the zero padding of the 112-feature rows), and 128 (they travel in a small shared-memory
+// array per slot); the packed head dims 32 and 64 and everything else take the FMA kernels.
+bool umma_rope_supported(const Problem& p) { return umma_supported(p) && (p.d == 112 || p.d == 128); }
 
 int umma_run(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
   if (p.N == 0 || (!c.k && !c.q)) return LINATTN_OK;
@@ -1451,7 +1462,7 @@ int umma_run(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t 
     case 32: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<32, false>(p, c, workspace, stream);
     case 64: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<64, false>(p, c, workspace, stream);
     case 112: return c.rope ? launch_fused<112, true>(p, c, workspace, stream) : launch_fused<112, false>(p, c, workspace, stream);
-    case 128: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<128, false>(p, c, workspace, stream);
+    case 128: return c.rope ? launch_fused<128, true>(p, c, workspace, stream) : launch_fused<128, false>(p, c, workspace, stream);
   }
   return LINATTN_ERR_UNSUPPORTED;
 }

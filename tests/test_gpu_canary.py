@@ -103,7 +103,8 @@ def test_forward_state_apply_stay_inside_their_buffers(la, dtype, H, d):
             assert torch.isfinite(o.float()).all() and la.workspace_status(wsr) == 0
 
 
-@pytest.mark.parametrize("dtype,H,d", [("bf16", 3, 112), ("bf16", 20, 112), ("bf16", 6, 64), ("f32", 2, 112), ("bf16", 3, 40)])
+@pytest.mark.parametrize("dtype,H,d", [("bf16", 3, 112), ("bf16", 20, 112), ("bf16", 6, 64), ("f32", 2, 112), ("bf16", 3, 40),
+                                       ("bf16", 5, 128)])
 def test_block_cache_calls_stay_inside_their_buffers(la, dtype, H, d):
     """step, peek, absorb, prefill (block by block and all blocks together), and the rotary forms, on blocks whose
     last one is short, with the cache's state and workspace between guard bands."""
