@@ -94,9 +94,15 @@ struct Cfg {
   // per SM the memory system's queues grow and the SMs' shares of the bandwidth drift apart.
   static constexpr int STATE_STAGES = DATA_BYTES / STAGE_BYTES < 4 ? DATA_BYTES / STAGE_BYTES : 4;
   static constexpr int BAR_BYTES = 1024;
-  // rotary variant without row padding (d = 128): the denominators of a tile's rows travel in a small array per slot
-  static constexpr int DEN_BYTES = D == 128 ? APPLY_SLOTS * kTileApply * 4 : 0;
-  static constexpr size_t SMEM = 1024 + DATA_BYTES + BAR_BYTES + DEN_BYTES;
+  // rotary variant without row padding (every head dim but 112): the denominators of a tile's rows travel in a small
+  // array per slot and head of the group
+  static constexpr int DEN_BYTES = D == 112 ? 0 : G * APPLY_SLOTS * kTileApply * 4;
+  static constexpr size_t SMEM = 1024 + DATA_BYTES + BAR_BYTES;
+  static constexpr size_t SMEM_ROPE = SMEM + DEN_BYTES;
+  // rotary variant: 16-byte chunk of a token's table row (d/2 fp16 pairs) that goes with logical chunk lc of box 0 / 1.
+  // With packed heads (d = 32, 64) box 1 starts a new head, so both boxes use the same chunk.
+  static constexpr bool SAME_TAB = 64 % D == 0;
+  __host__ __device__ static constexpr int tab_chunk(int box, int lc) { return ((64 * box + 8 * lc) % D) / 8; }
 };
 
 // How the (unit, token tile) work of one pass is dealt to the persistent grid.
@@ -387,10 +393,11 @@ __device__ __forceinline__ void reduce_elements(const FusedParams& p, int first,
       // behind the record (per warp, per feature): per warp slot the records in their fixed order, then the
       // slots as a balanced tree over sixteen, the missing ones zero (the association reduce_image's shuffles give)
       const int e = idx % E4;
-      const float4* zp = reinterpret_cast<const float4*>(p.partials) + E4 + (e - D * D / 4);
+      const int ft4 = (((idx / E4) % p.H) % C::G) * (D / 4) + (e - D * D / 4);   // float4 of the operand's 128 features
+      const float4* zp = reinterpret_cast<const float4*>(p.partials) + C::G * E4 + ft4;
       // (one slot after the other: this form only runs when the operand images are not in use, and the
       // rotary kernel has no registers to spare)
-      const bool upper = e - D * D / 4 >= 16;   // features 64..: the epilogue warps' slots hold a share too
+      const bool upper = ft4 >= 16;   // features 64..: the epilogue warps' slots hold a share too
       // (computed depth first, a few registers at a time: this form only runs when the operand images are not in
       // use, and the rotary kernel has no registers to spare)
       auto slot = [&](int w) {
@@ -690,7 +697,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   uint64_t* seg_done = s_ready + 1;        // every MMA of the finished segment is complete
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(seg_done + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
-  float* den_rows = reinterpret_cast<float*>(smem + C::DATA_BYTES + C::BAR_BYTES);   // [NSC][128], d = 128 with rotary factors
+  float* den_rows = reinterpret_cast<float*>(smem + C::DATA_BYTES + C::BAR_BYTES);   // [NSC][G][128]: rotary variant, every head dim but 112
   static_assert((3 * NSA + 5 + 4 * NSC + 6) * 8 + 8 <= C::BAR_BYTES, "barrier block too small");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -828,8 +835,11 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       tab0[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
       if (i == 0) tab1[0] = tab0[i];
       if (n < p.N) {
-        tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
-        if (i == 0 && box1_live) tab1[0] = __ldg(p.rope + n * (D / 8) + 8 + lc);
+        tab0[i] = __ldg(p.rope + n * (D / 8) + C::tab_chunk(0, lc));
+        if (i == 0) {
+          if (C::SAME_TAB) tab1[0] = tab0[0];
+          else if (box1_live) tab1[0] = __ldg(p.rope + n * (D / 8) + C::tab_chunk(1, lc));
+        }
       }
     };
     if (ROPE) {
@@ -920,7 +930,7 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     auto fetch_roth = [&](int tile, int j) {
       const long long n = (long long)tile * kTileState + 32 + row0h + 16 * j;
       tabh[j] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
-      if (h_live && n < p.N) tabh[j] = __ldg(p.rope + n * (D / 8) + 8 + lch);
+      if (h_live && n < p.N) tabh[j] = __ldg(p.rope + n * (D / 8) + C::tab_chunk(1, lch));
     };
     if (ROPE) {
       TileWalk t0(wa);
@@ -1108,8 +1118,9 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       const long long n = (long long)tile * kTileApply + row0 + 32 * i;
       tab0[i] = tab1[i] = make_uint4(kRopeIdentity, kRopeIdentity, kRopeIdentity, kRopeIdentity);
       if (n < p.N) {
-        tab0[i] = __ldg(p.rope + n * (D / 8) + lc);
-        if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + 8 + lc);
+        tab0[i] = __ldg(p.rope + n * (D / 8) + C::tab_chunk(0, lc));
+        if (C::SAME_TAB) tab1[i] = tab0[i];
+        else if (box1_live) tab1[i] = __ldg(p.rope + n * (D / 8) + C::tab_chunk(1, lc));
       }
     };
     if (ROPE) {
@@ -1138,12 +1149,19 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
           build_s_operand<D>(s_op, p.state, u / p.HG, u % p.HG, p.H, tr, R::RELU_THREADS + 128);
         }
         if (ROPE) {
-          const float4* zrow = reinterpret_cast<const float4*>(p.state + ((size_t)u * (D + 1) + D) * D);  // G = 1: unit = (b, h)
-          const float4 a0 = __ldcg(zrow + 2 * lc), a1 = __ldcg(zrow + 2 * lc + 1);
-          zc[0] = make_float2(a0.x, a0.y); zc[1] = make_float2(a0.z, a0.w); zc[2] = make_float2(a1.x, a1.y); zc[3] = make_float2(a1.z, a1.w);
-          if (box1_live) {
-            const float4 b0 = __ldcg(zrow + 16 + 2 * lc), b1 = __ldcg(zrow + 16 + 2 * lc + 1);
-            zc[4] = make_float2(b0.x, b0.y); zc[5] = make_float2(b0.z, b0.w); zc[6] = make_float2(b1.x, b1.y); zc[7] = make_float2(b1.z, b1.w);
+          // feature 64 * box + 8 * lc of the operand is feature fl of head g of the group
+#pragma unroll
+          for (int box = 0; box < 2; ++box) {
+            const int f0 = 64 * box + 8 * lc, g = f0 / D, fl = f0 - g * D;
+            const int h = (u % p.HG) * C::G + g;
+            float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+            if ((box == 0 || box1_live) && h < p.H) {
+              const float4* zrow = reinterpret_cast<const float4*>(p.state + ((size_t)((u / p.HG) * p.H + h) * (D + 1) + D) * D);
+              a0 = __ldcg(zrow + fl / 4);
+              a1 = __ldcg(zrow + fl / 4 + 1);
+            }
+            zc[4 * box + 0] = make_float2(a0.x, a0.y); zc[4 * box + 1] = make_float2(a0.z, a0.w);
+            zc[4 * box + 2] = make_float2(a1.x, a1.y); zc[4 * box + 3] = make_float2(a1.z, a1.w);
           }
         }
         if (!(C::G == 1 && p.s_image)) {
@@ -1170,21 +1188,46 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
           for (int e = 0; e < 4; ++e) den2 = fma2(f[e], zc[e], den2);
           *c0 = rotate_pack8(f, tab0[i]);
           uint4* c1 = reinterpret_cast<uint4*>(p0 + HALF + i * 32 * kRowBytes);
+          float2 den2b = make_float2(0.f, 0.f);   // packed heads: box 1 belongs to other heads than box 0
           if (box1_live) {
             unpack_relu8(*c1, f);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) den2 = fma2(f[e], zc[4 + e], den2);
+            for (int e = 0; e < 4; ++e) {
+              if (C::G == 1) den2 = fma2(f[e], zc[4 + e], den2);
+              else den2b = fma2(f[e], zc[4 + e], den2b);
+            }
             *c1 = rotate_pack8(f, tab1[i]);
           }
           float den = den2.x + den2.y;
           if (!tn.done()) fetch_rot(tn.tile(), i);  // this row's rotations for the next tile
-          den += __shfl_xor_sync(0xffffffffu, den, 1);
-          den += __shfl_xor_sync(0xffffffffu, den, 2);
-          den += __shfl_xor_sync(0xffffffffu, den, 4);
-          if (D == 112) {
-            if (lc == 6) *reinterpret_cast<float*>(c1) = den;  // chunk 6 of the second box: features 112..119
+          // The eight lanes of a row hold one chunk of each box.  One head per operand: add all of it over the eight.
+          // Packed heads: box 1 belongs to other heads, and with d = 32 a head is four lanes wide; the first exchange
+          // hands one box's sum to the partner lane, so that each half of the lanes reduces one box.
+          const int row = row0 + 32 * i;
+          if (C::G == 1) {
+            den += __shfl_xor_sync(0xffffffffu, den, 1);
+            den += __shfl_xor_sync(0xffffffffu, den, 2);
+            den += __shfl_xor_sync(0xffffffffu, den, 4);
+            if (D == 112) {
+              if (lc == 6) *reinterpret_cast<float*>(c1) = den;  // chunk 6 of the second box: features 112..119
+            } else {
+              if (pc == 0) den_rows[s * kTileApply + row] = den;   // no padding to carry it
+            }
           } else {
-            if (pc == 0) den_rows[s * kTileApply + row0 + 32 * i] = den;   // no padding to carry it
+            const float denb = den2b.x + den2b.y;
+            constexpr int XB = C::G == 2 ? 4 : 2;             // lane bit that picks the box after the exchange
+            const bool second = (pc & XB) != 0;
+            float x = second ? denb : den;
+            x += __shfl_xor_sync(0xffffffffu, second ? den : denb, XB);
+            x += __shfl_xor_sync(0xffffffffu, x, 1);
+            if (C::G == 2) x += __shfl_xor_sync(0xffffffffu, x, 2);
+            // d = 64: lane 0 of the row has head 0 (box 0), lane 4 head 1.  d = 32: lanes with the same pc / 4 share
+            // a head, whose place in its box is lc / 4; lanes 0 and 4 have box 0, lanes 2 and 6 box 1
+            if (C::G == 2) {
+              if ((pc & 3) == 0) den_rows[(s * 2 + (second ? 1 : 0)) * kTileApply + row] = x;
+            } else {
+              if ((pc & 1) == 0) den_rows[(s * 4 + (second ? 2 : 0) + (lc >> 2)) * kTileApply + row] = x;
+            }
           }
         }
         fence_proxy_async_smem();
@@ -1224,9 +1267,12 @@ umma_fused_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       float rinv[C::G];
       if (ROPE) {
         // the ReLU warps left phi(q) . z of this row in the row's padding
-        const float den = D == 112 ? *reinterpret_cast<const float*>(sl + HALF + r * kRowBytes + ((6 ^ (r & 7)) << 4))
-                                   : den_rows[s * kTileApply + r];
-        rinv[0] = 1.0f / (den + p.eps);
+        if (D == 112) {
+          rinv[0] = 1.0f / (*reinterpret_cast<const float*>(sl + HALF + r * kRowBytes + ((6 ^ (r & 7)) << 4)) + p.eps);
+        } else {
+#pragma unroll
+          for (int g = 0; g < C::G; ++g) rinv[g] = 1.0f / (den_rows[(s * C::G + g) * kTileApply + r] + p.eps);
+        }
       } else {
         uint32_t dn[4];
         tmem_ld_x4(trow + C::ZROW, dn);
@@ -1420,17 +1466,18 @@ int launch_fused(const Problem& p, const UmmaCall& c, void* workspace, cudaStrea
   if (!do_state) { mk = mq; mv = mq; }
   // the opt-in to more than 48 KB of dynamic shared memory is a per-device setting of the kernel
   static bool attr_set[64] = {false};
+  constexpr size_t kSmem = ROPE ? C::SMEM_ROPE : C::SMEM;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LINATTN_ERR_CUDA;
   if (!attr_set[dev]) {
-    if (cudaFuncSetAttribute(umma_fused_kernel<D, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM) !=
+    if (cudaFuncSetAttribute(umma_fused_kernel<D, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem) !=
         cudaSuccess)
       return LINATTN_ERR_CUDA;
     attr_set[dev] = true;
   }
   void* args[] = {&mk, &mv, &mq, &mo, &fp};
   const cudaError_t e = cudaLaunchCooperativeKernel((const void*)umma_fused_kernel<D, ROPE>, dim3(grid), dim3(Roles<ROPE>::THREADS), args,
-                                                    C::SMEM, stream);
+                                                    kSmem, stream);
   if (e != cudaSuccess) { cudaGetLastError(); return LINATTN_ERR_CUDA; }
   count_launches(1);
   return LINATTN_OK;
@@ -1451,16 +1498,17 @@ size_t umma_partial_bytes(const Problem& p, bool rope) {
   return ((size_t)kMaxCtas + units) * (G * (size_t)p.state_elems() + (rope ? kZParts : 0)) * sizeof(float);
 }
 
-// The rotary variant runs on the tensor cores at the one-head-per-operand head dims: 112, the paper's (the
-// denominators travel in the zero padding of the 112-feature rows), and 128 (they travel in a small shared-memory
-// array per slot); the packed head dims 32 and 64 and everything else take the FMA kernels.
-bool umma_rope_supported(const Problem& p) { return umma_supported(p) && (p.d == 112 || p.d == 128); }
+// The rotary variant runs on the tensor cores wherever the plain kernel does.  d = 112, the paper's: the denominators
+// travel in the zero padding of the 112-feature rows; every other head dim: in a small shared-memory array per slot
+// and head of the group.  With packed heads (d = 32, 64) both boxes of a row use the same 16-byte chunk of the
+// rotation table, since box 1 starts a new head.  Everything else takes the FMA kernels.
+bool umma_rope_supported(const Problem& p) { return umma_supported(p); }
 
 int umma_run(const Problem& p, const UmmaCall& c, void* workspace, cudaStream_t stream) {
   if (p.N == 0 || (!c.k && !c.q)) return LINATTN_OK;
   switch (p.d) {
-    case 32: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<32, false>(p, c, workspace, stream);
-    case 64: return c.rope ? LINATTN_ERR_UNSUPPORTED : launch_fused<64, false>(p, c, workspace, stream);
+    case 32: return c.rope ? launch_fused<32, true>(p, c, workspace, stream) : launch_fused<32, false>(p, c, workspace, stream);
+    case 64: return c.rope ? launch_fused<64, true>(p, c, workspace, stream) : launch_fused<64, false>(p, c, workspace, stream);
     case 112: return c.rope ? launch_fused<112, true>(p, c, workspace, stream) : launch_fused<112, false>(p, c, workspace, stream);
     case 128: return c.rope ? launch_fused<128, true>(p, c, workspace, stream) : launch_fused<128, false>(p, c, workspace, stream);
   }

@@ -124,7 +124,7 @@ def test_random_walk_rotary(la, orc, seed):
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     check = assert_parity_f32
     if dtype == "bf16":   # the tensor-core path rounds the rotated queries and keys to bf16 as well
-        check = lambda got, ref, what: assert_parity_bf16(got, ref, what, rms_rel=1.5e-2 if d in (112, 128) else 1e-2)
+        check = lambda got, ref, what: assert_parity_bf16(got, ref, what, rms_rel=1.5e-2 if d in (32, 64, 112, 128) else 1e-2)
     N = sum(lens)
     q, k, v = (synth.gauss((B, N, H, d), seed, t, dtype=dtype) for t in (1, 2, 3))
     theta = synth.gauss((N, d // 2), seed, 7, dtype="f32").astype(np.float64) * 3.0
@@ -155,7 +155,7 @@ def test_random_walk_rotary(la, orc, seed):
         ref = orc.rope_block_step(ocache, *blk_h, cs[sl], sn[sl], EPS)
         if o is not None:
             check(to_f64(o), ref, what)
-        # the tensor-core path (bf16, d = 112 or 128) rounds the rotated keys to bf16 before the MMA
-        state_close(to_f64(cache.state), *ocache, 1e-2 if (dtype == "bf16" and d in (112, 128)) else 1e-5, what)
+        # the tensor-core path (bf16, d = 32, 64, 112 or 128) rounds the rotated keys to bf16 before the MMA
+        state_close(to_f64(cache.state), *ocache, 1e-2 if (dtype == "bf16" and d in (32, 64, 112, 128)) else 1e-5, what)
         n0 += T
     assert cache.info()["blocks_seen"] == len(lens) and cache.status() == 0

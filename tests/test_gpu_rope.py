@@ -34,6 +34,9 @@ SHAPES = [
     (1, (2, 7, 11), 2, 128),
     (2, (4, 9, 20), 5, 128),     # tensor-core path at d = 128: several tiles, trailing CTAs, a ragged tail
     (2, (3, 5, 7), 5, 64),
+    (2, (4, 9, 20), 5, 64),      # packed heads on the tensor cores: two per operand, an odd head count, a ragged tail
+    (1, (5, 10, 20), 7, 32),     # four per operand, the last group with three heads
+    (2, (2, 7, 11), 9, 32),
     (1, (2, 5, 9), 3, 6),
 ]
 
@@ -77,7 +80,8 @@ def test_rope_errors(la):
 
 
 @pytest.mark.parametrize("case", [("bf16", 3, 112, (7, 6, 10), 60), ("f32", 2, 112, (4, 5, 5), 25), ("bf16", 2, 64, (6, 4, 8), 64),
-                                  ("bf16", 2, 112, (3, 1, 150), 150), ("bf16", 3, 128, (5, 7, 9), 130)],
+                                  ("bf16", 2, 112, (3, 1, 150), 150), ("bf16", 3, 128, (5, 7, 9), 130), ("bf16", 6, 32, (6, 4, 8), 64),
+                                  ("bf16", 3, 64, (5, 7, 9), 130)],
                          ids=lambda c: "%s_H%d_d%d_Tb%d" % (c[0], c[1], c[2], c[4]))
 def test_rope_block_steps_match_the_block_causal_oracle(la, orc, case):
     """Cached block-by-block generation with rotary factors against the oracle's block-causal form; the last
@@ -120,7 +124,7 @@ def packed_table(la, T, Hh, Ww, d):
     return table, packed[..., 0], packed[..., 1]
 
 
-@pytest.mark.parametrize("dtype,d", [("bf16", 112), ("f32", 112), ("bf16", 64), ("bf16", 6), ("bf16", 128)])
+@pytest.mark.parametrize("dtype,d", [("bf16", 112), ("f32", 112), ("bf16", 64), ("bf16", 6), ("bf16", 128), ("bf16", 32)])
 def test_rope_denoise_loop_reads_without_committing(la, orc, dtype, d):
     """Algorithm 1 on the attention the model runs (Eq. 2 with RoPE): every denoising step of a block reads the
     rotary cache together with the noisy block itself and leaves the cache as it was; only the clean block is
@@ -154,7 +158,7 @@ def test_rope_denoise_loop_reads_without_committing(la, orc, dtype, d):
         # z sums the plain features in fp32.  S sums rotated features: fp32 throughout on the fp32 path; on the bf16
         # path the rotated key is rounded to bf16 before it enters the tensor core (2^-9 relative per term, unbiased:
         # the sum's error is about 1.5e-3 of the state's RMS, its largest of 37 632 entries several times that)
-        for g, r, name, rel in ((got[..., :d, :].swapaxes(-1, -2), S, "S", 1e-2 if (dtype == "bf16" and d in (112, 128)) else 1e-5),
+        for g, r, name, rel in ((got[..., :d, :].swapaxes(-1, -2), S, "S", 1e-2 if (dtype == "bf16" and d in (32, 64, 112, 128)) else 1e-5),
                                 (got[..., d, :], z, "z", 1e-5)):
             rms = np.sqrt((r ** 2).mean(axis=tuple(range(2, r.ndim)), keepdims=True))
             assert (np.abs(g - r) <= rel * (np.abs(r) + rms)).all(), f"rotary cache after block {blk}: {name}"
@@ -162,7 +166,7 @@ def test_rope_denoise_loop_reads_without_committing(la, orc, dtype, d):
 
 
 @pytest.mark.parametrize("case", [("bf16", 3, 112, (6, 6, 10), 2), ("f32", 2, 112, (4, 5, 5), 1), ("bf16", 2, 64, (6, 4, 8), 3),
-                                  ("bf16", 2, 6, (4, 3, 5), 2), ("bf16", 4, 128, (6, 5, 9), 2)],
+                                  ("bf16", 2, 6, (4, 3, 5), 2), ("bf16", 4, 128, (6, 5, 9), 2), ("bf16", 5, 32, (6, 4, 8), 2)],
                          ids=lambda c: "%s_H%d_d%d_fb%d" % (c[0], c[1], c[2], c[4]))
 def test_rope_prefill_equals_steps_and_oracle(la, orc, case):
     """blocklin_prefill_rope over all blocks: the bits of single rotary steps, the oracle's block-causal rotary form,
