@@ -581,6 +581,18 @@ def extras(torch, la, synth, dev, peak):
         res[w.name] = {"H": w.H, "d": w.d, "ms": ms, "tokens_heads_per_s": w.B * w.N * w.H / (ms * 1e-3),
                        "algorithmic_gbs": by / (ms * 1e-3) / 1e9, "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak,
                        "l2": "one input set of %.0f MB (> 126 MB L2)" % (by / 1e6)}
+        # the same layer with the rotary factors of Eq. 2 (3D table over the 21 x 45 x 80 latent grid)
+        cos, sin = synth.rope_table(21, 45, 80, w.d)
+        table = la.rope_pack(torch.from_numpy(cos).to(dev), torch.from_numpy(sin).to(dev))
+        wsr = la.new_rope_workspace(q)
+        for _ in range(3):
+            la.linattn_forward_rope(q, k, v, table, w.eps, out=o, workspace=wsr)
+        ms = time_loop(torch, lambda i: la.linattn_forward_rope(q, k, v, table, w.eps, out=o, workspace=wsr), n) / n
+        res[w.name + "_rope"] = {"H": w.H, "d": w.d, "ms": ms, "tokens_heads_per_s": w.B * w.N * w.H / (ms * 1e-3),
+                                 "algorithmic_gbs": by / (ms * 1e-3) / 1e9, "frac_of_peak": by / (ms * 1e-3) / 1e9 / peak,
+                                 "note": "q,k,v,o bytes only; the fp16 rotation table (%.1f MB) is re-read from L2 by every "
+                                         "tensor-core operand" % (table.numel() * 2 / 1e6)}
+        del table, wsr, cos, sin
         if w.d == 112:
             # the same layer with head-major memory ([B,H,N,d] behind the same [B,N,H,d] view): a head's rows are
             # then contiguous instead of 224 bytes out of every 4480
